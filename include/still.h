@@ -1,0 +1,205 @@
+/*
+ * still.h -- C ABI of the STILL intra-layer hybrid attention layer forward for
+ * NVIDIA B200 (sm_100a).
+ *
+ * The layer (paper Sec. 3, "Methodology") takes the per-head queries, keys and
+ * values of one attention layer and, for every query token t,
+ *   1. computes the Self-Saliency Score of every token from sliding-window
+ *      attention over the last C tokens (Sec. 3.1, Eqs. diag / nodiag / score),
+ *   2. keeps, per chunk of C tokens, the top-k (the paper's lambda) scoring
+ *      tokens for softmax attention; selection is delayed: a chunk is routed
+ *      when it leaves the two-chunk local region (Sec. 3.3, Eq.
+ *      delayed_selection),
+ *   3. folds every other token of a routed chunk into a linear-attention state
+ *      (s, z) through the Norm-Preserved Feature Map (Sec. 3.2, Eq.
+ *      feature_map; Sec. 3.3, Eq. cache_routing_sum),
+ *   4. outputs y_t = (N_SA + N_LA) / (D_SA + D_LA) (Sec. 3.3, merge equation and
+ *      the definitions of N_SA, D_SA, N_LA, D_LA).
+ * still_hybrid_attn_fwd is the chunk-wise parallel form (Algorithm 1) used for
+ * prefill; still_hybrid_attn_step is the recurrent form (Sec. 3.3) used for
+ * decode.  Both are defined per head; with grouped KV heads, query head h uses
+ * KV head h / (H / Hkv) and scores, selection and state are per query head.
+ *
+ * General conventions
+ *   - Every tensor pointer is DEVICE memory owned by the caller, contiguous in
+ *     the stated layout, aligned to 16 bytes.  The library allocates no device
+ *     memory and keeps no global state.
+ *   - Calls enqueue work on `cuda_stream` (a cudaStream_t passed as void*, NULL =
+ *     the legacy default stream) and return without synchronising.
+ *   - Return value: STILL_OK (0) or a negative still_status code.  No C++
+ *     exception crosses this boundary.  There is no CPU fallback: a call either
+ *     runs the CUDA kernels or fails.
+ *   - Device-side waits (mbarrier waits inside the tensor-core kernels) are
+ *     bounded; if one expires the kernel records a code in the status word at
+ *     the start of the workspace, drains, frees its tensor memory and returns.
+ *     still_device_status reads that word.
+ */
+#ifndef STILL_H_
+#define STILL_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum still_status {
+    STILL_OK = 0,
+    STILL_ERR_INVALID_ARG = -1,      /* null pointer, bad shape, topk > chunk, H % Hkv != 0, misaligned pointer */
+    STILL_ERR_UNSUPPORTED = -2,      /* shape or dtype outside what the kernels cover (see still_params_t)     */
+    STILL_ERR_WORKSPACE_TOO_SMALL = -3,
+    STILL_ERR_STATE_FULL = -4,       /* decode state has no room for another token                             */
+    STILL_ERR_CUDA = -5,             /* a CUDA runtime / driver call failed (launch error, no sm_100 device)    */
+    STILL_ERR_DEVICE_TIMEOUT = -6,   /* a bounded device-side wait expired (reported by still_device_status)    */
+    STILL_ERR_STATE_MISMATCH = -7    /* decode state was built with other parameters                            */
+} still_status;
+
+enum { STILL_DTYPE_FP32 = 0, STILL_DTYPE_BF16 = 1 };
+
+/*
+ * Problem description (Algorithm 1, "Input": q, k, v, gate g, feature maps
+ * phi_q / phi_k, chunk size C, number lambda, small constant epsilon).
+ *
+ * Supported: d in {64, 128}; d_f in {32, 64, 128} with d_f <= d; chunk in
+ * {64, 128}; 0 <= topk <= chunk; dtype fp32 or bf16.  bf16 inputs run on the
+ * tcgen05 tensor-core kernels, fp32 inputs on fp32 FMA kernels (TF32 would not
+ * meet the 1e-4 output tolerance).
+ */
+typedef struct still_params {
+    int32_t B;          /* batch                                                             */
+    int32_t H;          /* query heads                                                       */
+    int32_t Hkv;        /* KV heads, H % Hkv == 0                                            */
+    int32_t d;          /* head dim                                                          */
+    int32_t d_f;        /* width of the NP-Map linear map f; the feature dim is d' = 2 d_f   */
+    int32_t chunk;      /* C: chunk size = score window w                                    */
+    int32_t topk;       /* lambda: tokens kept for softmax attention per chunk               */
+    int32_t dtype;      /* STILL_DTYPE_*: type of Q, K, V, G, Wq, bq, Wk, bk, Y               */
+    float sm_scale;     /* multiplies q.k in the score and in the SA branch (1 = the main     */
+                        /* text's exp(qk^T); d^-1/2 = App. A.1, Eq. softmax_attention)       */
+    float eps;          /* epsilon of the Self-Saliency Score                                */
+    int64_t max_salient;/* reserved, must be 0: the salient cache is unbounded (Eq.          */
+                        /* cache_routing_sum as written)                                      */
+} still_params_t;
+
+/* Bytes of workspace still_hybrid_attn_fwd needs for a sequence of N tokens
+ * (0 if the parameters are invalid).  Host-only arithmetic, no CUDA call. */
+size_t still_workspace_bytes(const still_params_t *p, int64_t N);
+
+/* Bytes of a decode state that can hold up to max_tokens tokens per sequence
+ * (0 if the parameters are invalid).  Host-only arithmetic.  Layout: see
+ * still_state_layout_t below. */
+size_t still_state_bytes(const still_params_t *p, int64_t max_tokens);
+
+/*
+ * Byte offsets of the parts of a decode state, so that a caller can inspect,
+ * copy or checkpoint it (the state is a plain buffer; copying it is a
+ * checkpoint).  Fills *out and returns STILL_OK, or an error for bad parameters.
+ *   header   : 256 bytes, int32 words {magic, version, B, H, Hkv, d, d_f, chunk,
+ *              topk, dtype, capacity_lo, capacity_hi, t_lo, t_hi, status, 0...};
+ *              t = tokens consumed so far.
+ *   k_cache, v_cache : [B, Hkv, capacity, d] in dtype -- the K/V history
+ *              (local region + every earlier token; the salient pairs of Eq.
+ *              cache_routing_sum are rows of it named by sel_idx).
+ *   score    : [B, H, capacity] fp32 -- Self-Saliency Score of every token.
+ *   sel_idx  : [B, H, capacity / chunk, topk] int32 -- salient positions of each
+ *              routed chunk, ascending, -1 padded (rows of chunks not yet routed
+ *              are unspecified).
+ *   S        : [B, H, 2 d_f, d] fp32 -- KV state s_t.
+ *   z        : [B, H, 2 d_f] fp32 -- normaliser z_t.
+ *   scratch  : split-KV partial results of the step kernel.
+ */
+typedef struct still_state_layout {
+    size_t header, k_cache, v_cache, score, sel_idx, S, z, scratch, total;
+    int64_t capacity; /* max_tokens rounded up to a multiple of chunk */
+} still_state_layout_t;
+int still_state_layout(const still_params_t *p, int64_t max_tokens, still_state_layout_t *out);
+
+/*
+ * Prefill: Algorithm 1 (Chunk-Wise Parallel Form) over N tokens.
+ *
+ *   Q        [B, H, N, d]     queries
+ *   K, V     [B, Hkv, N, d]   keys, values
+ *   G        [B, H, N, d]     gate values g_t (already activated) or NULL = ones;
+ *                             multiplies N_LA only
+ *   Wq, bq   [H, d, d_f], [H, d_f] or NULL      f of phi_q: f(x) = x Wq + bq
+ *   Wk, bk   [Hkv, d, d_f], [Hkv, d_f] or NULL  f of phi_k
+ *   Y        [B, H, N, d]     output, or NULL to skip the SA branch and the merge
+ *                             (useful when only state_out is wanted)
+ *   scores   [B, H, N] fp32   Self-Saliency Scores, or NULL
+ *   sel_idx  [B, H, ceil(N/chunk), topk] int32: absolute positions of the selected
+ *            tokens of every chunk, ascending, -1 padded when a ragged last chunk
+ *            has fewer than topk tokens; or NULL (a workspace copy is used)
+ *   state_out  decode state of still_state_bytes(p, max_tokens) bytes with
+ *            capacity >= N, or NULL.  On return it describes the sequence after N
+ *            tokens, ready for still_hybrid_attn_step with t_pos = N.
+ *   state_max_tokens  the max_tokens the state was sized with (ignored if
+ *            state_out is NULL)
+ *   workspace, workspace_bytes  at least still_workspace_bytes(p, N)
+ *
+ * Ties in the score are broken by position (smaller first); NaN scores rank
+ * lowest.  N need not be a multiple of chunk.  N = 0 is a no-op.
+ * Errors: STILL_ERR_INVALID_ARG, STILL_ERR_UNSUPPORTED,
+ * STILL_ERR_WORKSPACE_TOO_SMALL, STILL_ERR_STATE_FULL (N > capacity),
+ * STILL_ERR_CUDA.
+ */
+int still_hybrid_attn_fwd(const still_params_t *p, int64_t N, const void *Q, const void *K,
+                          const void *V, const void *G, const void *Wq, const void *bq,
+                          const void *Wk, const void *bk, void *Y, float *scores, int32_t *sel_idx,
+                          void *state_out, int64_t state_max_tokens, void *workspace,
+                          size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Decode: one step of the Recurrent Form (Sec. 3.3) for every sequence of the
+ * batch.  t_pos is the number of tokens the state already holds (the new token
+ * gets 0-based position t_pos); the caller tracks it on the host and it must
+ * match the state (a mismatch is recorded in the state's status word).
+ *
+ *   q [B, H, d], k, v [B, Hkv, d], g [B, H, d] or NULL, y [B, H, d]
+ *   Wq, bq, Wk, bk as for the prefill
+ *
+ * The step appends (k, v), scores the new token, routes the chunk that has just
+ * left the two-chunk local region when the new token opens a chunk (top-k into
+ * sel_idx, the rest into S and z), and writes y by the merge equation.
+ * Errors: STILL_ERR_INVALID_ARG, STILL_ERR_UNSUPPORTED, STILL_ERR_STATE_FULL
+ * (t_pos >= capacity), STILL_ERR_CUDA.
+ */
+int still_hybrid_attn_step(const still_params_t *p, void *state, int64_t state_max_tokens,
+                           int64_t t_pos, const void *q, const void *k, const void *v,
+                           const void *g, const void *Wq, const void *bq, const void *Wk,
+                           const void *bk, void *y, void *cuda_stream);
+
+/*
+ * Prefill with HOST buffers: copies Q, K, V (and G, the NP-Map parameters) from
+ * host memory (pinned memory makes the copies asynchronous) into `arena`, runs
+ * still_hybrid_attn_fwd and copies Y (and scores / sel_idx when not NULL) back.
+ * `arena` is device memory of at least still_host_arena_bytes(p, N) bytes; it
+ * holds the staged tensors and the workspace.  The call returns after
+ * synchronising the stream, so the host outputs are valid on return.
+ */
+size_t still_host_arena_bytes(const still_params_t *p, int64_t N);
+int still_hybrid_attn_fwd_host(const still_params_t *p, int64_t N, const void *hQ, const void *hK,
+                               const void *hV, const void *hG, const void *hWq, const void *hbq,
+                               const void *hWk, const void *hbk, void *hY, float *hscores,
+                               int32_t *hsel_idx, void *arena, size_t arena_bytes,
+                               void *cuda_stream);
+
+/*
+ * Reads the device status word of a workspace (prefill) or of a decode state
+ * after synchronising `cuda_stream`.  *status receives STILL_OK or
+ * STILL_ERR_DEVICE_TIMEOUT / STILL_ERR_STATE_MISMATCH; *detail (optional)
+ * receives a kernel-specific code saying which wait gave up.
+ */
+int still_device_status(const void *workspace_or_state, void *cuda_stream, int *status, int *detail);
+
+/* Number of kernel launches the last still_hybrid_attn_fwd / _step call on this
+ * host thread enqueued (for launch accounting in benchmarks). */
+int still_last_launch_count(void);
+
+/* Static string for a status code. */
+const char *still_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* STILL_H_ */

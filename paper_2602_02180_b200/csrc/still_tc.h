@@ -1,0 +1,29 @@
+// Internal interfaces between the host API (still_api.cu), the tensor-core
+// prefill kernels (still_tc.cu) and the decode-step kernels (still_step.cu).
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/still.h"
+
+namespace still {
+
+// ---- tensor-core (tcgen05) prefill path, bf16 only --------------------------------
+// True when the softmax-attention branch of these parameters runs on the tcgen05 kernel.
+bool tc_supported(const still_params_t *p);
+// Rows per head of the compacted salient K/V copies (selected rows of all chunks plus tile padding).
+long long tc_sel_rows(const still_params_t *p, long long N);
+// Compacts the selected K/V rows and runs the softmax-attention + merge kernel.
+int tc_sa_merge(const still_params_t *p, long long N, const void *Q, const void *K, const void *V,
+                const int32_t *sel_idx, const float *N_LA, const float *D_LA, void *Y, void *k_sel,
+                void *v_sel, long long sel_rows, int *status_words, cudaStream_t st, int *launches);
+
+// ---- decode step ----------------------------------------------------------------------
+size_t step_scratch_bytes(const still_params_t *p, long long capacity);
+int step_launch(const still_params_t *p, char *state, const still_state_layout_t *L, long long t_pos,
+                const void *q, const void *k, const void *v, const void *g, const void *Wq,
+                const void *bq, const void *Wk, const void *bk, void *y, cudaStream_t st,
+                int *launches);
+
+}  // namespace still

@@ -1,0 +1,118 @@
+"""Parity of the CUDA prefill (still_hybrid_attn_fwd, through the C ABI) with the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2602_02180_b200 as still
+from paper_2602_02180_b200 import synth
+from tests import util_parity as U
+
+pytestmark = pytest.mark.gpu
+
+
+def _small(name, dtype, B, H, Hkv, d, N, C, k, recipe="iid", seed=1):
+    return synth.Workload(name, B, H, Hkv, d, N, C, k, dtype, recipe, 4242 + seed)
+
+
+def test_c1_fp32_every_row():
+    w = synth.WORKLOADS["c1"]
+    r = U.run_prefill(w)
+    heads = U.sample_heads(w, 99)
+    U.check_selection(r["scores"], r["sel"], w.C, w.k, heads)
+    worst, serr = U.check_outputs(w, r["Q"], r["K"], r["V"], r["Wq"], r["Wk"], r["Y"], r["scores"], r["sel"], heads)
+    assert serr < 1e-4
+    print(f"c1 max-abs {worst:.2e} score err {serr:.2e}")
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize(
+    "B,H,Hkv,d,N,C,k",
+    [
+        (1, 2, 1, 64, 200, 32, 8),      # ragged tail, GQA
+        (2, 4, 2, 64, 64 * 5 + 17, 64, 16),
+        (1, 4, 4, 128, 128 * 3 + 1, 128, 32),
+        (1, 2, 2, 64, 300, 64, 0),      # lambda = 0: local softmax + linear attention
+        (1, 2, 1, 128, 333, 64, 1),
+        (1, 2, 2, 64, 260, 64, 64),     # lambda = C: causal softmax attention
+        (1, 2, 1, 128, 40, 64, 16),     # shorter than one chunk
+        (1, 1, 1, 64, 1, 32, 4),        # a single token
+        (1, 8, 2, 128, 128 * 4, 128, 128),
+    ],
+)
+def test_small_shapes(dtype, B, H, Hkv, d, N, C, k):
+    w = _small("t", dtype, B, H, Hkv, d, N, C, k)
+    r = U.run_prefill(w, gate=True, bias=True)
+    heads = U.sample_heads(w, 4)
+    if k:
+        U.check_selection(r["scores"], r["sel"], C, k, heads)
+    U.check_outputs(w, r["Q"], r["K"], r["V"], r["Wq"], r["Wk"], r["Y"], r["scores"], r["sel"], heads,
+                    G=r["G"], bq=r["bq"], bk=r["bk"])
+
+
+def test_paper_literal_scale_one():
+    # sm_scale = 1 is the main text's exp(q k^T); inputs are scaled down so the softmaxes stay soft.
+    w = _small("t", "fp32", 1, 2, 2, 64, 256, 64, 16)
+    Q, K, V = synth.make_qkv(w, "cuda")
+    Q, K = Q * 0.35, K * 0.35
+    Wq, Wk = synth.make_npmap_weights(w, "cuda")
+    p = still.StillParams(w.B, w.H, w.Hkv, w.d, w.C, w.k, torch.float32, sm_scale=1.0)
+    Y, scores, sel = still.hybrid_attn_fwd(p, Q, K, V, Wq, Wk)
+    heads = U.sample_heads(w, 2)
+    U.check_selection(scores, sel, w.C, w.k, heads)
+    from oracle import still_oracle as oracle
+    for b, h in heads:
+        out = oracle.chunkwise(U.f64(Q[b, h]), U.f64(K[b, h]), U.f64(V[b, h]), U.f64(Wq[h]), U.f64(Wk[h]),
+                               oracle.HeadParams(w.C, w.k, 1.0), forced_idx=sel[b, h].cpu().numpy())
+        assert np.abs(U.f64(Y[b, h]) - out["y"]).max() < 1e-4
+
+
+def test_run_to_run_determinism():
+    w = _small("t", "bf16", 1, 4, 2, 64, 500, 64, 16)
+    a = U.run_prefill(w)
+    b = U.run_prefill(w)
+    assert torch.equal(a["Y"], b["Y"]) and torch.equal(a["sel"], b["sel"]) and torch.equal(a["scores"], b["scores"])
+
+
+def test_constant_value_rows():
+    # y is a positive-weight average of the values: constant V gives constant y (gate = 1).
+    w = _small("t", "fp32", 1, 2, 2, 64, 320, 64, 16)
+    Q, K, V = synth.make_qkv(w, "cuda")
+    V = torch.ones_like(V) * 0.75
+    Wq, Wk = synth.make_npmap_weights(w, "cuda")
+    Y, _, _ = still.hybrid_attn_fwd(U.params_of(w), Q, K, V, Wq, Wk)
+    assert (Y - 0.75).abs().max().item() < 1e-5
+
+
+def test_c2_sampled():
+    w = synth.WORKLOADS["c2"]
+    r = U.run_prefill(w)
+    heads = U.sample_heads(w, 6, seed=2)
+    rows = U.sample_rows(w.N, 96, w.C, seed=2)
+    U.check_selection(r["scores"], r["sel"], w.C, w.k, heads)
+    worst, serr = U.check_outputs(w, r["Q"], r["K"], r["V"], r["Wq"], r["Wk"], r["Y"], r["scores"], r["sel"],
+                                  heads, rows=rows)
+    print(f"c2 max-abs {worst:.2e} score err {serr:.2e}")
+    # companion with a non-degenerate selection (lambda = C/4)
+    w4 = w.with_(k=w.C // 4)
+    r = U.run_prefill(w4)
+    U.check_selection(r["scores"], r["sel"], w4.C, w4.k, heads)
+    U.check_outputs(w4, r["Q"], r["K"], r["V"], r["Wq"], r["Wk"], r["Y"], r["scores"], r["sel"], heads, rows=rows)
+
+
+def test_invalid_arguments_are_rejected():
+    w = _small("t", "bf16", 1, 2, 2, 64, 128, 64, 16)
+    Q, K, V = synth.make_qkv(w, "cuda")
+    Wq, Wk = synth.make_npmap_weights(w, "cuda")
+    p = U.params_of(w)
+    with pytest.raises(still.StillError) as e:
+        still.hybrid_attn_fwd(p, Q, K, V, Wq, Wk, workspace=torch.empty(1024, dtype=torch.uint8, device="cuda"))
+    assert e.value.code == -3
+    bad = still.StillParams(1, 3, 2, 64, 64, 16)
+    assert still.workspace_bytes(bad, 128) == 0
+    with pytest.raises(still.StillError):
+        still.hybrid_attn_fwd(still.StillParams(1, 2, 2, 64, 64, 65), Q, K, V, Wq, Wk,
+                              workspace=torch.empty(1 << 20, dtype=torch.uint8, device="cuda"))
+    ws = torch.empty(still.workspace_bytes(p, 128) + 16, dtype=torch.uint8, device="cuda")
+    with pytest.raises(still.StillError) as e:  # misaligned workspace pointer
+        still.hybrid_attn_fwd(p, Q, K, V, Wq, Wk, workspace=ws[1:])
+    assert e.value.code == -1
