@@ -1,0 +1,403 @@
+#!/usr/bin/env python
+"""Benchmark of the STILL hybrid attention layer forward on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c3] [--impl ours|reference]
+
+One "step" is one still_hybrid_attn_fwd call (score -> top-k select -> NP-Map + linear scan ->
+sparse softmax attention -> merge) over one synthetic batch of the workload; for the decode
+workload (c5) a step is one still_hybrid_attn_step call.  The metric is tokens/s/layer
+(B * N / time).  With N GPUs every rank runs its own batch (the (batch, head) units are
+independent: no collective on the data path) and the value is the sum over ranks divided by the
+slowest rank's time.
+
+The JSON line carries, besides the contract keys:
+  roofline      the softmax-attention kernel (>98% of the FLOPs): algorithmic FLOPs per launch
+                divided by its CUDA-event time measured inside the timed region, against the
+                measured bf16 peak of this machine (MEASURED_PEAKS.json, sustained figure)
+  cpu_baseline  the CPU oracle timed on a bounded sample of the same workload on this machine
+  e2e           the same metric through still_hybrid_attn_fwd_host with pinned HOST buffers
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "hybrid-attn prefill tokens/s/layer at Llama-3-8B shape"
+UNIT = "tokens/s"
+
+
+def algorithmic_work(w, lam=None):
+    """FLOPs and bytes the method itself needs for one prefill call (causal-exact pair count)."""
+    lam = w.k if lam is None else lam
+    C, d, N = w.C, w.d, w.N
+    T = -(-N // C)
+    BH, BHkv = w.B * w.H, w.B * w.Hkv
+    es = 4 if w.dtype == "fp32" else 2
+    p_sel = C * lam * max(T - 1, 0) * max(T - 2, 0) // 2
+    p_loc = max(T - 1, 0) * C * C + T * C * (C + 1) // 2
+    f_sa = 4 * d * (p_sel + p_loc) * BH
+    dp = 2 * w.d_f
+    la = lam < C
+    f_map = 2 * d * w.d_f * N * (BH + BHkv) if la else 0
+    f_la = (2 * (C - lam) + 2 * C) * dp * (d + 1) * max(T - 2, 0) * BH if la else 0
+    f_score = 2 * d * (2 * C) * C * T * BH  # s_in and s_prev tiles
+    by = w.B * N * d * es * (2 * w.H + 2 * w.Hkv) + 4 * BH * N + 4 * BH * T * lam
+    return {"flops": f_sa + f_map + f_la + f_score, "flops_sa": f_sa, "bytes": by}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index=0):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 7:
+                continue
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"bf16_tflops": p["bf16_tflops"], "bf16_tflops_sustained": p["bf16_tflops_sustained"],
+                "hbm_gbs": p["hbm_gbs"], "source": "measured"}
+    return {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0, "source": "fallback"}
+
+
+def ncu_traffic(kernel_key):
+    """DRAM bytes per launch of the dominant kernel from the committed ncu summary, if any."""
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(path):
+        return json.load(open(path)).get(kernel_key)
+    return None
+
+
+def oracle_sample(w, lam, n_heads, n_rows, seed=0):
+    """Times the CPU oracle on a bounded sample: n_heads heads in parallel, all O(N) steps in full,
+    the softmax/merge step on n_rows evenly spread query rows; returns the extrapolated time of
+    the whole workload, the threads used and a description of the sample."""
+    import numpy as np
+    import torch
+
+    from oracle import still_oracle as oracle
+    from paper_2602_02180_b200 import synth
+
+    ws = w.with_(B=1, H=n_heads, Hkv=n_heads, k=lam)
+    Q, K, V = synth.make_qkv(ws, "cpu")
+    Wq, Wk = synth.make_npmap_weights(ws, "cpu")
+    f64 = lambda t: t.float().numpy().astype(np.float64)  # noqa: E731
+    Q, K, V, Wq, Wk = map(f64, (Q, K, V, Wq, Wk))
+    hp = oracle.HeadParams(w.C, lam, w.sm_scale)
+    rows = np.unique(np.linspace(0, w.N - 1, n_rows).astype(np.int64))
+    t0 = time.perf_counter()
+    out = oracle.layer(Q, K, V, Wq, Wk, hp, rows=rows[-1:])
+    t_fixed = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    out = oracle.layer(Q, K, V, Wq, Wk, hp, rows=rows)
+    t_rows = time.perf_counter() - t0
+    threads = out["threads"]
+    per_row = max(t_rows - t_fixed, 1e-9) / max(len(rows) - 1, 1)
+    per_head_batch = t_fixed + per_row * w.N  # n_heads heads processed side by side
+    total = per_head_batch * (w.B * w.H) / n_heads
+    sample = (f"{n_heads} of {w.B * w.H} heads on {threads} threads; score/select/state steps in full, "
+              f"softmax+merge on {len(rows)} of {w.N} query rows, scaled by row and head count")
+    return total, threads, sample, t_fixed + t_rows
+
+
+def run_reference(args, w, lam, rank, world):
+    """--impl reference: the CPU oracle as it stands, on this machine's host cores."""
+    if rank != 0:
+        return
+    import multiprocessing
+
+    cores = multiprocessing.cpu_count()
+    n_heads = max(1, min(cores, w.B * w.H))
+    n_rows = 48 if w.N > 8192 else 256
+    times = []
+    for i in range(args.warmup + args.steps):
+        total, threads, sample, spent = oracle_sample(w, lam, n_heads, n_rows)
+        if i >= args.warmup:
+            times.append(total)
+    t = statistics.mean(times)
+    value = w.B * w.N / t
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "H": w.H, "Hkv": w.Hkv, "d": w.d, "N": w.N, "chunk": w.C,
+                   "topk": lam, "timing": "host wall clock, extrapolated from a bounded sample"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c3", choices=["c1", "c2", "c3", "c4", "c5"])
+    ap.add_argument("--topk", type=int, default=None, help="override lambda (e.g. the C/4 companion)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+
+    from paper_2602_02180_b200 import synth
+
+    w = synth.WORKLOADS[args.workload]
+    lam = w.k if args.topk is None else args.topk
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        run_reference(args, w, lam, rank, world)
+        return
+
+    import torch
+
+    import paper_2602_02180_b200 as still
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the CUDA library has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    dev = torch.device("cuda", local_rank)
+
+    if w.name == "c5":
+        line = bench_decode(args, w, lam, still, synth, torch, dist, dev, rank, world)
+    else:
+        line = bench_prefill(args, w, lam, still, synth, torch, dist, dev, rank, world)
+    if rank == 0:
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def _barrier(torch, dist):
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+
+
+def _max_over_ranks(torch, dist, x, dev):
+    if dist is None:
+        return x
+    t = torch.tensor([x], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def bench_prefill(args, w, lam, still, synth, torch, dist, dev, rank, world):
+    wl = w.with_(k=lam, seed=w.seed + 100 * rank)
+    Q, K, V = synth.make_qkv(wl, dev)
+    Wq, Wk = synth.make_npmap_weights(wl, dev)
+    p = still.StillParams(w.B, w.H, w.Hkv, w.d, w.C, lam, w.torch_dtype)
+    Y = torch.empty_like(Q)
+    T = -(-w.N // w.C)
+    scores = torch.empty(w.B, w.H, w.N, dtype=torch.float32, device=dev)
+    sel = torch.empty(w.B, w.H, T, max(lam, 1), dtype=torch.int32, device=dev)
+    ws = torch.empty(still.workspace_bytes(p, w.N), dtype=torch.uint8, device=dev)
+    call = lambda: still.hybrid_attn_fwd(p, Q, K, V, Wq, Wk, Y=Y, scores=scores, sel_idx=sel, workspace=ws)  # noqa: E731
+
+    for _ in range(max(args.warmup, 3)):
+        call()
+    launches_per_step = still.last_launch_count()
+    _barrier(torch, dist)
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    still.profile_enable(args.steps)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        call()
+    e1.record()
+    _barrier(torch, dist)
+    ms_total = e0.elapsed_time(e1)
+    kernel_ms = still.profile_collect()
+    clocks = sampler.stop() if rank == 0 else None
+    ms_total = _max_over_ranks(torch, dist, ms_total, dev)
+    assert still.device_status(ws) == (0, 0), "a device-side wait timed out"
+    ms_step = ms_total / args.steps
+    value = world * w.B * w.N / (ms_step * 1e-3)
+
+    work = algorithmic_work(w, lam)
+    peaks = measured_peaks()
+    k_ms = statistics.mean(kernel_ms) if kernel_ms else None
+    fp32 = w.dtype == "fp32"
+    roof = None
+    if k_ms:
+        ach = work["flops_sa"] / (k_ms * 1e-3) / 1e12
+        peak = peaks["bf16_tflops_sustained"]
+        roof = {"bound": "tensor", "kernel": "softmax-attention + merge", "achieved": ach, "peak": peak,
+                "unit": "TFLOP/s", "frac": ach / peak, "peak_source": peaks["source"] + " (sustained cuBLAS bf16)",
+                "frac_of_burst_peak": ach / peaks["bf16_tflops"], "frac_of_nominal_2250": ach / 2250.0,
+                "kernel_ms": k_ms, "kernel_share_of_step": k_ms / ms_step,
+                "traffic": ncu_traffic(f"sa_{w.name}_k{lam}"),
+                "whole_step_frac_of_nominal_roofline": (work["flops"] / 2.25e15) / (ms_step * 1e-3)}
+        if fp32:
+            roof["bound"] = "alu"
+            roof["note"] = "fp32 inputs run on FMA pipes; peak shown is the bf16 tensor peak for context"
+
+    e2e = None
+    if not args.no_e2e:
+        hQ, hK, hV = (t.cpu().pin_memory() for t in (Q, K, V))
+        hWq, hWk = Wq.cpu().pin_memory(), Wk.cpu().pin_memory()
+        hY = torch.empty_like(hQ).pin_memory()
+        arena = torch.empty(still.host_arena_bytes(p, w.N), dtype=torch.uint8, device=dev)
+        n_e2e = max(2, min(args.steps, 5))
+        still.hybrid_attn_fwd_host(p, hQ, hK, hV, hWq, hWk, hY=hY, arena=arena)
+        _barrier(torch, dist)
+        t0 = time.perf_counter()
+        e0.record()
+        for _ in range(n_e2e):
+            still.hybrid_attn_fwd_host(p, hQ, hK, hV, hWq, hWk, hY=hY, arena=arena)
+        e1.record()
+        _barrier(torch, dist)
+        ms_e2e = max(e0.elapsed_time(e1), (time.perf_counter() - t0) * 1e3) / n_e2e
+        ms_e2e = _max_over_ranks(torch, dist, ms_e2e, dev)
+        h2d = sum(t.numel() * t.element_size() for t in (hQ, hK, hV, hWq, hWk))
+        d2h = hY.numel() * hY.element_size()
+        e2e = {"value": world * w.B * w.N / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e, "steps": n_e2e}
+        del arena, hQ, hK, hV, hY
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import multiprocessing
+
+        n_heads = max(1, min(multiprocessing.cpu_count(), w.B * w.H))
+        total, threads, sample, _ = oracle_sample(w, lam, n_heads, 48 if w.N > 8192 else 256)
+        cpu = {"value": w.B * w.N / total, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample}
+
+    return {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16" if not fp32 else "f32", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "H": w.H, "Hkv": w.Hkv, "d": w.d, "N": w.N, "chunk": w.C,
+                   "topk": lam, "l2": "inputs larger than L2 (no flush)", "per_gpu_batch": w.B},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
+        "roofline": roof, "cpu_baseline": cpu,
+        "algorithmic": {"flops_per_step": work["flops"], "bytes_per_step": work["bytes"]},
+    }
+
+
+def bench_decode(args, w, lam, still, synth, torch, dist, dev, rank, world):
+    """c5: the prefix is summarised into a decode state by the prefill, then `steps` decode steps
+    are timed.  HBM-bound: the salient K/V history is read once per KV head per step."""
+    p = still.StillParams(w.B, w.H, w.Hkv, w.d, w.C, lam, w.torch_dtype)
+    n_steps = args.steps
+    cap = w.N + max(n_steps, w.steps) + args.warmup + 8
+    state = torch.zeros(still.state_bytes(p, cap), dtype=torch.uint8, device=dev)
+    Wq, Wk = synth.make_npmap_weights(w, dev)
+    wl = w.with_(seed=w.seed + 100 * rank)
+    Q, K, V = synth.make_qkv(wl, dev)
+    ws = torch.empty(still.workspace_bytes(p, w.N), dtype=torch.uint8, device=dev)
+    still.hybrid_attn_fwd(p, Q, K, V, Wq, Wk, state=state, state_max_tokens=cap, workspace=ws, want_y=False)
+    del Q, K, V, ws
+    torch.cuda.synchronize()
+    t = w.N
+    ins = [synth.make_decode_inputs(wl, i, dev) for i in range(8)]
+    y = torch.empty(w.B, w.H, w.d, dtype=w.torch_dtype, device=dev)
+    for i in range(max(args.warmup, 3)):
+        q, k, v = ins[i % 8]
+        still.hybrid_attn_step(p, state, cap, t, q, k, v, Wq, Wk, y=y)
+        t += 1
+    launches = still.last_launch_count()
+    _barrier(torch, dist)
+    sampler = ClockSampler(dev.index or 0)
+    if rank == 0:
+        sampler.start()
+    still.profile_enable(n_steps)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(n_steps):
+        q, k, v = ins[i % 8]
+        still.hybrid_attn_step(p, state, cap, t, q, k, v, Wq, Wk, y=y)
+        t += 1
+    e1.record()
+    _barrier(torch, dist)
+    ms_total = _max_over_ranks(torch, dist, e0.elapsed_time(e1), dev)
+    kernel_ms = still.profile_collect()
+    clocks = sampler.stop() if rank == 0 else None
+    assert still.device_status(state)[0] == 0
+    ms_step = ms_total / n_steps
+    peaks = measured_peaks()
+    es = 2
+    n_hist = (t // w.C - 1) * lam if lam > 0 else 0
+    # K and V rows of the salient history once per KV head, the local region, and the LA state
+    by = w.B * w.Hkv * (n_hist + 2 * w.C) * w.d * es * 2 + (w.B * w.H * 2 * w.d_f * (w.d + 1) * 4 if lam < w.C else 0)
+    k_ms = statistics.mean(kernel_ms) if kernel_ms else ms_step
+    ach = by / (k_ms * 1e-3) / 1e9
+    roof = {"bound": "hbm", "kernel": "split-KV attend", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+            "frac": ach / peaks["hbm_gbs"], "peak_source": peaks["source"], "kernel_ms": k_ms,
+            "traffic": ncu_traffic(f"attend_{w.name}_k{lam}")}
+    return {
+        "metric": "hybrid-attn decode tokens/s/layer at Llama-3-8B shape", "value": world * w.B / (ms_step * 1e-3),
+        "unit": UNIT, "n_gpus": world, "steps": n_steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "H": w.H, "Hkv": w.Hkv, "d": w.d, "prefix": w.N, "chunk": w.C,
+                   "topk": lam, "l2": "K/V history larger than L2 (no flush)"},
+        "clocks": clocks, "e2e": None, "gpu_launches": launches * n_steps, "roofline": roof, "cpu_baseline": None,
+    }
+
+
+if __name__ == "__main__":
+    main()

@@ -196,6 +196,19 @@ int still_device_status(const void *workspace_or_state, void *cuda_stream, int *
  * host thread enqueued (for launch accounting in benchmarks). */
 int still_last_launch_count(void);
 
+/*
+ * Optional timing of the dominant kernel (the softmax-attention + merge kernel of the
+ * prefill, the split-KV attend kernel of the decode step) for roofline reports.
+ * still_profile_enable(n) creates n pairs of CUDA events owned by the library (host
+ * objects, no device memory); from then on every call on this host thread records one
+ * pair around that kernel on the caller's stream, until n pairs are used.
+ * still_profile_collect synchronises the recorded events, writes the elapsed
+ * milliseconds of each pair to ms[0..*n_records) (at most `capacity`), destroys the
+ * events and disables the timing.  Not for use during stream capture.
+ */
+int still_profile_enable(int max_records);
+int still_profile_collect(float *ms, int capacity, int *n_records);
+
 /* Static string for a status code. */
 const char *still_strerror(int status);
 

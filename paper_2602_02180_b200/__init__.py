@@ -8,6 +8,8 @@ from .binding import (  # noqa: F401
     hybrid_attn_fwd_host,
     hybrid_attn_step,
     last_launch_count,
+    profile_collect,
+    profile_enable,
     state_bytes,
     state_layout,
     strerror,

@@ -94,6 +94,10 @@ def lib():
         L.still_device_status.restype = ctypes.c_int
         L.still_device_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_int)]
         L.still_last_launch_count.restype = ctypes.c_int
+        L.still_profile_enable.restype = ctypes.c_int
+        L.still_profile_enable.argtypes = [ctypes.c_int]
+        L.still_profile_collect.restype = ctypes.c_int
+        L.still_profile_collect.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.c_int, ctypes.POINTER(ctypes.c_int)]
         L.still_strerror.restype = ctypes.c_char_p
         L.still_strerror.argtypes = [ctypes.c_int]
         _lib = L
@@ -204,6 +208,22 @@ def hybrid_attn_fwd_host(p: StillParams, hQ, hK, hV, hWq=None, hWk=None, hG=None
     if rc != STILL_OK:
         raise StillError(rc, "still_hybrid_attn_fwd_host")
     return hY
+
+
+def profile_enable(max_records: int) -> None:
+    rc = lib().still_profile_enable(max_records)
+    if rc != STILL_OK:
+        raise StillError(rc, "still_profile_enable")
+
+
+def profile_collect(capacity: int = 4096) -> list[float]:
+    """Milliseconds of the dominant kernel for every call since profile_enable."""
+    buf = (ctypes.c_float * capacity)()
+    n = ctypes.c_int(0)
+    rc = lib().still_profile_collect(buf, capacity, ctypes.byref(n))
+    if rc != STILL_OK:
+        raise StillError(rc, "still_profile_collect")
+    return [buf[i] for i in range(n.value)]
 
 
 def device_status(buf) -> tuple[int, int]:

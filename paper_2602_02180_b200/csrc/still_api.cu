@@ -17,6 +17,20 @@ namespace still {
 
 static thread_local int g_launches = 0;
 
+// Event pairs of still_profile_enable (per host thread).
+static thread_local cudaEvent_t *g_prof_ev = nullptr;
+static thread_local int g_prof_cap = 0, g_prof_used = 0;
+
+void profile_mark_begin(cudaStream_t st) {
+    if (g_prof_ev && g_prof_used < g_prof_cap) cudaEventRecord(g_prof_ev[2 * g_prof_used], st);
+}
+void profile_mark_end(cudaStream_t st) {
+    if (g_prof_ev && g_prof_used < g_prof_cap) {
+        cudaEventRecord(g_prof_ev[2 * g_prof_used + 1], st);
+        ++g_prof_used;
+    }
+}
+
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 static inline size_t esize(int dtype) { return dtype == STILL_DTYPE_FP32 ? 4 : 2; }
 
@@ -251,7 +265,9 @@ static int fwd_typed(const still_params_t *p, long long N, const T *Q, const T *
             rc = tc_sa_merge(p, N, Q, K, V, sel, nla, dla, Y, ws + w.ksel, ws + w.vsel, w.sel_rows,
                              reinterpret_cast<int *>(ws + w.status), st, &g_launches);
         } else {
+            profile_mark_begin(st);
             rc = launch_sa_merge<T>(p, N, w.T, Q, K, V, sel, nla, dla, Y, st);
+            profile_mark_end(st);
         }
         if (rc != STILL_OK) return rc;
     }
@@ -448,6 +464,40 @@ int still_device_status(const void *workspace_or_state, void *cuda_stream, int *
 }
 
 int still_last_launch_count(void) { return g_launches; }
+
+int still_profile_enable(int max_records) {
+    if (max_records <= 0 || g_prof_ev) return STILL_ERR_INVALID_ARG;
+    g_prof_ev = new cudaEvent_t[2 * (size_t)max_records];
+    for (int i = 0; i < 2 * max_records; ++i)
+        if (cudaEventCreate(&g_prof_ev[i]) != cudaSuccess) {
+            for (int j = 0; j < i; ++j) cudaEventDestroy(g_prof_ev[j]);
+            delete[] g_prof_ev;
+            g_prof_ev = nullptr;
+            return STILL_ERR_CUDA;
+        }
+    g_prof_cap = max_records;
+    g_prof_used = 0;
+    return STILL_OK;
+}
+
+int still_profile_collect(float *ms, int capacity, int *n_records) {
+    if (!g_prof_ev || !ms || !n_records) return STILL_ERR_INVALID_ARG;
+    int rc = STILL_OK, n = 0;
+    for (int i = 0; i < g_prof_used; ++i) {
+        float t = 0.f;
+        if (cudaEventSynchronize(g_prof_ev[2 * i + 1]) != cudaSuccess ||
+            cudaEventElapsedTime(&t, g_prof_ev[2 * i], g_prof_ev[2 * i + 1]) != cudaSuccess)
+            rc = STILL_ERR_CUDA;
+        else if (n < capacity)
+            ms[n++] = t;
+    }
+    for (int i = 0; i < 2 * g_prof_cap; ++i) cudaEventDestroy(g_prof_ev[i]);
+    delete[] g_prof_ev;
+    g_prof_ev = nullptr;
+    g_prof_cap = g_prof_used = 0;
+    *n_records = n;
+    return rc;
+}
 
 const char *still_strerror(int status) {
     switch (status) {

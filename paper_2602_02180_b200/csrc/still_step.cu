@@ -359,12 +359,14 @@ static int step_typed(const still_params_t *p, char *state, const still_state_la
     }
     const long long cps = n_routed > 0 ? (n_routed + n_splits - 1) / n_splits : 1;
     dim3 grid(n_splits + 1, p->Hkv, p->B);
+    profile_mark_begin(st);
     if (d == 64)
         step_attend_kernel<T, 2><<<grid, 128, 0, st>>>(kc, vc, sel, q, part, p->H, p->Hkv, cap, C, lam, t,
                                                        n_splits, cps, n_routed, p->sm_scale);
     else
         step_attend_kernel<T, 4><<<grid, 128, 0, st>>>(kc, vc, sel, q, part, p->H, p->Hkv, cap, C, lam, t,
                                                        n_splits, cps, n_routed, p->sm_scale);
+    profile_mark_end(st);
     ++*launches;
     STILL_CUDA(cudaGetLastError());
 

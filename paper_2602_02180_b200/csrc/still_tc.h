@@ -9,6 +9,10 @@
 
 namespace still {
 
+// ---- timing of the dominant kernel (still_profile_enable / still_profile_collect) ----
+void profile_mark_begin(cudaStream_t st);
+void profile_mark_end(cudaStream_t st);
+
 // ---- tensor-core (tcgen05) prefill path, bf16 only --------------------------------
 // True when the softmax-attention branch of these parameters runs on the tcgen05 kernel.
 bool tc_supported(const still_params_t *p);
