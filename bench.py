@@ -260,7 +260,7 @@ def bench_prefill(args, w, lam, still, synth, torch, dist, dev, rank, world):
         call()
     launches_per_step = still.last_launch_count()
     _barrier(torch, dist)
-    sampler = ClockSampler(local_rank)
+    sampler = ClockSampler(dev.index or 0)
     if rank == 0:
         sampler.start()
     still.profile_enable(args.steps)
