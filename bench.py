@@ -188,6 +188,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c3", choices=["c1", "c2", "c3", "c4", "c5"])
     ap.add_argument("--topk", type=int, default=None, help="override lambda (e.g. the C/4 companion)")
+    ap.add_argument("--B", type=int, default=None, help="override the batch (profiling of a smaller case)")
+    ap.add_argument("--H", type=int, default=None, help="override the query heads (KV heads scale along)")
+    ap.add_argument("--N", type=int, default=None, help="override the sequence length")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -196,6 +199,9 @@ def main():
     from paper_2602_02180_b200 import synth
 
     w = synth.WORKLOADS[args.workload]
+    if args.B or args.H or args.N:
+        H = args.H or w.H
+        w = w.with_(B=args.B or w.B, H=H, Hkv=max(1, H * w.Hkv // w.H), N=args.N or w.N)
     lam = w.k if args.topk is None else args.topk
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))

@@ -1,14 +1,672 @@
-// Tensor-core (tcgen05) prefill path -- placeholder until the kernel lands.
+// Tensor-core prefill path for bf16 (sm_100a): salient K/V compaction and the
+// softmax-attention + merge kernel on tcgen05 / TMEM / TMA.
+//
+// Softmax Attention Branch of Algorithm 1 + the merge equation of Sec. 3.3.
+// For a query in chunk c the keys are: the selected tokens of chunks 0..c-2, all
+// of chunk c-1, and chunk c up to the query itself.  The selected rows of every
+// chunk are first compacted per query head into K_sel / V_sel ([B*H, sel_rows, d],
+// ascending position), so that "selected tokens of chunks 0..c-2" is the prefix
+// [0, (c-1)*lambda) of a contiguous array that TMA can tile.
+//
+// One CTA owns 256 consecutive query rows of one (batch, head): two query tiles
+// A and B of 128 rows, each with its own S accumulator (128 fp32 columns of TMEM)
+// and O accumulator (d columns).  The key stream of the CTA is a sequence of
+// 128-key tiles: SEL tiles j (rows [128j, 128j+128) of K_sel / V_sel) followed by
+// the three LOC tiles (rows of K / V at positions [128m, 128m+128), m = m0-1, m0,
+// m0+1 with m0 = first row / 128).  Which columns of a tile a query row sees is a
+// per-row column interval, applied as a mask in the softmax.
+//
+// Warp roles (384 threads):
+//   warp 0     TMA producer: Q tiles once, then K and V tiles through mbarrier rings
+//   warp 1     MMA issuer (one elected thread): S_X = Q_X K^T (operands in shared
+//              memory, SWIZZLE_128B K-major), O_X += P_X V (P_X read from TMEM, V in
+//              shared memory MN-major); tcgen05.commit signals the softmax warps and
+//              frees the ring stages
+//   warps 4-7  softmax of tile A: one thread per query row (tcgen05.ld of the S row),
+//              online softmax in the log2 domain with lazy rescaling of O, P written
+//              back to TMEM as bf16 over S
+//   warps 8-11 the same for tile B
+//   The softmax warps also run the epilogue: O / l merged with the linear branch
+//   (N_LA, D_LA) under one denominator and stored as bf16.
+//
+// Every mbarrier wait is bounded: on expiry the kernel records
+// STILL_ERR_DEVICE_TIMEOUT in the status word, all roles leave their loops, and
+// tensor memory is freed before the CTA exits.
 #include "still_tc.h"
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include <algorithm>
+
+#include "still_common.cuh"
 
 namespace still {
 
-bool tc_supported(const still_params_t *) { return false; }
-long long tc_sel_rows(const still_params_t *, long long) { return 0; }
-int tc_sa_merge(const still_params_t *, long long, const void *, const void *, const void *,
-                const int32_t *, const float *, const float *, void *, void *, void *, long long, int *,
-                cudaStream_t, int *) {
-    return STILL_ERR_UNSUPPORTED;
+namespace {
+
+constexpr int kBlockM = 128;   // query rows per tile
+constexpr int kBlockN = 128;   // keys per tile
+constexpr int kThreads = 384;
+constexpr long long kWaitLimitCycles = 4000000000ll;  // ~2 s at 2 GHz
+
+// ----------------------------------------------------------------- PTX wrappers
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false (and flags the CTA as aborted) when the limit expires
+// or another role has already aborted.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag,
+                                          int *status, int where) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    int spins = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++spins & 1023) == 0) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > kWaitLimitCycles) {
+                *abort_flag = 1;
+                report_status(status, STILL_ERR_DEVICE_TIMEOUT, where);
+                return false;
+            }
+        }
+    }
+    return true;
+}
+__device__ __forceinline__ void fence_barrier_init() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, uint64_t *bar, int x, int y) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t *dst_smem, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)),
+                 "r"(ncols)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() {
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after() {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_commit(uint64_t *bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+// D[tmem] (+)= A[smem desc] * B[smem desc]
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                       uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem desc]
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                       uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+#define STILL_R32(r, o)                                                                               \
+    "=r"(r[o + 0]), "=r"(r[o + 1]), "=r"(r[o + 2]), "=r"(r[o + 3]), "=r"(r[o + 4]), "=r"(r[o + 5]),     \
+    "=r"(r[o + 6]), "=r"(r[o + 7]), "=r"(r[o + 8]), "=r"(r[o + 9]), "=r"(r[o + 10]), "=r"(r[o + 11]),  \
+    "=r"(r[o + 12]), "=r"(r[o + 13]), "=r"(r[o + 14]), "=r"(r[o + 15]), "=r"(r[o + 16]),              \
+    "=r"(r[o + 17]), "=r"(r[o + 18]), "=r"(r[o + 19]), "=r"(r[o + 20]), "=r"(r[o + 21]),              \
+    "=r"(r[o + 22]), "=r"(r[o + 23]), "=r"(r[o + 24]), "=r"(r[o + 25]), "=r"(r[o + 26]),              \
+    "=r"(r[o + 27]), "=r"(r[o + 28]), "=r"(r[o + 29]), "=r"(r[o + 30]), "=r"(r[o + 31])
+
+// 32 consecutive fp32 columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t *r) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : STILL_R32(r, 0)
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t *r) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]),
+        "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]),
+        "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+// Shared-memory matrix descriptor (SWIZZLE_128B, 8-row groups 1024 bytes apart).
+// lbo_bytes: distance between 64-element atoms along the MN dimension (MN-major
+// operands only; ignored for K-major operands with swizzling).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3ffff) >> 4);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3fff) << 16;
+    d |= (uint64_t)((1024 >> 4) & 0x3fff) << 32;  // stride between 8-row groups
+    d |= (uint64_t)1 << 46;                         // descriptor version of sm_100
+    d |= (uint64_t)2 << 61;                         // SWIZZLE_128B
+    return d;
+}
+// Instruction descriptor of kind::f16 with bf16 operands and fp32 accumulation.
+__host__ __device__ constexpr uint32_t make_idesc(int M, int N, bool b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(N >> 3) << 17) |
+           ((uint32_t)(M >> 4) << 24);
+}
+
+// ----------------------------------------------------------------- shared memory plan
+
+template <int D>
+struct SmemPlan {
+    static constexpr int kTileBytes = kBlockN * D * 2;        // one K or V or Q tile
+    static constexpr int kKStages = (D == 128) ? 3 : 4;
+    static constexpr int kVStages = (D == 128) ? 2 : 3;
+    static constexpr int kQ = 0;                               // two Q tiles
+    static constexpr int kK = kQ + 2 * kTileBytes;
+    static constexpr int kV = kK + kKStages * kTileBytes;
+    static constexpr int kBar = kV + kVStages * kTileBytes;    // mbarriers
+    static constexpr int kNumBars = 1 + 2 * kKStages + 2 * kVStages + 6;
+    static constexpr int kMisc = kBar + kNumBars * 8;          // tmem base, abort flag
+    static constexpr int kTotal = kMisc + 16;
+    static constexpr int kAlloc = kTotal + 1024;               // slack to align the base to 1024
+};
+
+// Per-CTA description of the key stream.
+struct Stream {
+    int n_sel_a, n_sel_b;   // SEL tiles used by tile A / tile B
+    int m0;                 // first LOC tile index of interest is m0 - 1
+    int has_prev;           // m0 > 0
+    int has_b;              // tile B has rows below N
+    int n_tiles;            // stream length
+    // stream index i: [0, n_sel_b) SEL(i); then LOC(m0-1) (if has_prev), LOC(m0), LOC(m0+1) (if has_b)
+    __device__ __forceinline__ bool is_sel(int i) const { return i < n_sel_b; }
+    __device__ __forceinline__ int loc_m(int i) const { return m0 - has_prev + (i - n_sel_b); }
+    __device__ __forceinline__ bool used_by(int x, int i) const {
+        if (i < n_sel_b) return x == 0 ? (i < n_sel_a) : true;
+        int m = loc_m(i);
+        return x == 0 ? (m <= m0) : (m >= m0);
+    }
+};
+
+__device__ __forceinline__ int sel_limit(long long pos, int C, int lam) {  // visible prefix of K_sel
+    long long c = pos / C;
+    return c >= 2 ? (int)((c - 1) * lam) : 0;
+}
+
+template <int D>
+__global__ void __launch_bounds__(kThreads, 1)
+sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                   const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_ksel,
+                   const __grid_constant__ CUtensorMap tm_vsel, const float *__restrict__ N_LA,
+                   const float *__restrict__ D_LA, __nv_bfloat16 *__restrict__ Y, int *status, int H, int Hkv,
+                   int N, int C, int lam, int sel_rows, float scale_log2, int n_qblocks) {
+    using P = SmemPlan<D>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + P::kBar);
+    uint64_t *q_full = bars;
+    uint64_t *k_full = bars + 1, *k_empty = k_full + P::kKStages;
+    uint64_t *v_full = k_empty + P::kKStages, *v_empty = v_full + P::kVStages;
+    uint64_t *s_full = v_empty + P::kVStages;  // [2]
+    uint64_t *p_full = s_full + 2;             // [2]
+    uint64_t *o_final = p_full + 2;            // [2]
+    uint32_t *tmem_base_slot = reinterpret_cast<uint32_t *>(smem + P::kMisc);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + P::kMisc + 8);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int qb = n_qblocks - 1 - blockIdx.x;  // heavy blocks first
+    const int bh = blockIdx.y, b = bh / H, h = bh % H, kvh = h / (H / Hkv);
+    const int R0 = qb * 2 * kBlockM;
+
+    Stream st;
+    st.m0 = R0 / kBlockN;
+    st.has_prev = st.m0 > 0;
+    st.has_b = (R0 + kBlockM) < N;
+    {
+        int last_a = min(R0 + kBlockM - 1, N - 1), last_b = min(R0 + 2 * kBlockM - 1, N - 1);
+        st.n_sel_a = (sel_limit(last_a, C, lam) + kBlockN - 1) / kBlockN;
+        st.n_sel_b = st.has_b ? (sel_limit(last_b, C, lam) + kBlockN - 1) / kBlockN : st.n_sel_a;
+    }
+    st.n_tiles = st.n_sel_b + st.has_prev + 1 + st.has_b;
+
+    // A CTA that starts after another one has reported a failure does nothing.
+    if (threadIdx.x == 0) *abort_flag = *reinterpret_cast<volatile int *>(status) != 0;
+    __syncthreads();
+    if (*abort_flag) return;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        mbar_init(q_full, 1);
+        for (int i = 0; i < P::kKStages; ++i) { mbar_init(k_full + i, 1); mbar_init(k_empty + i, 2); }
+        for (int i = 0; i < P::kVStages; ++i) { mbar_init(v_full + i, 1); mbar_init(v_empty + i, 2); }
+        for (int i = 0; i < 2; ++i) { mbar_init(s_full + i, 1); mbar_init(p_full + i, 128); mbar_init(o_final + i, 1); }
+        *abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_base_slot, 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_base_slot;
+    // TMEM columns: S_A [0,128), S_B [128,256), O_A [256,256+D), O_B [256+D, 256+2D); P_X overlays S_X.
+    auto col_s = [](int x) -> uint32_t { return (uint32_t)x * 128u; };
+    auto col_o = [](int x) -> uint32_t { return 256u + (uint32_t)x * (uint32_t)D; };
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            const int q_row = bh * N + R0;
+            mbar_expect_tx(q_full, (st.has_b ? 2 : 1) * P::kTileBytes);
+            for (int x = 0; x < (st.has_b ? 2 : 1); ++x)
+                for (int half = 0; half < D / 64; ++half)
+                    tma_load_2d(smem + P::kQ + x * P::kTileBytes + half * (kBlockM * 128), &tm_q, q_full, half * 64,
+                                q_row + x * kBlockM);
+            bool ok = true;
+            int armed_k = 0, armed_v = 0;
+            for (int i = 0; i < st.n_tiles && ok; ++i) {
+                const bool sel = st.is_sel(i);
+                const CUtensorMap *mk = sel ? &tm_ksel : &tm_k, *mv = sel ? &tm_vsel : &tm_v;
+                const int row = sel ? bh * sel_rows + i * kBlockN : (b * Hkv + kvh) * N + st.loc_m(i) * kBlockN;
+                const int ks = i % P::kKStages, vs = i % P::kVStages;
+                ok = mbar_wait(k_empty + ks, ((i / P::kKStages) & 1) ^ 1, abort_flag, status, 1);
+                if (!ok) break;
+                mbar_expect_tx(k_full + ks, P::kTileBytes);
+                for (int half = 0; half < D / 64; ++half)
+                    tma_load_2d(smem + P::kK + ks * P::kTileBytes + half * (kBlockN * 128), mk, k_full + ks, half * 64, row);
+                armed_k = i + 1;
+                ok = mbar_wait(v_empty + vs, ((i / P::kVStages) & 1) ^ 1, abort_flag, status, 2);
+                if (!ok) break;
+                mbar_expect_tx(v_full + vs, P::kTileBytes);
+                for (int half = 0; half < D / 64; ++half)
+                    tma_load_2d(smem + P::kV + vs * P::kTileBytes + half * (kBlockN * 128), mv, v_full + vs, half * 64, row);
+                armed_v = i + 1;
+            }
+            if (!ok) {
+                // leave no copy in flight behind: wait (bounded) for the loads already issued
+                if (armed_k > 0) {
+                    int i = armed_k - 1;
+                    mbar_wait(k_full + i % P::kKStages, (i / P::kKStages) & 1, abort_flag, status, 3);
+                }
+                if (armed_v > 0) {
+                    int i = armed_v - 1;
+                    mbar_wait(v_full + i % P::kVStages, (i / P::kVStages) & 1, abort_flag, status, 3);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc_qk = make_idesc(kBlockM, kBlockN, false);
+            constexpr uint32_t idesc_pv = make_idesc(kBlockM, D, true);
+            bool ok = mbar_wait(q_full, 0, abort_flag, status, 4);
+            tc_fence_after();
+            int pending[2] = {-1, -1};   // stream tile whose P V product is still to be issued
+            int n_done[2] = {0, 0};      // tiles processed per query tile (phase of p_full)
+            auto issue_pv = [&](int x, int ip) -> bool {
+                if (!mbar_wait(p_full + x, n_done[x] & 1, abort_flag, status, 5)) return false;
+                const int vs = ip % P::kVStages;
+                if (!mbar_wait(v_full + vs, (ip / P::kVStages) & 1, abort_flag, status, 6)) return false;
+                tc_fence_after();
+                const uint32_t v_addr = smem_u32(smem + P::kV + vs * P::kTileBytes);
+#pragma unroll
+                for (int k = 0; k < kBlockN / 16; ++k)
+                    mma_ts(tmem_base + col_o(x), tmem_base + col_s(x) + k * 8,
+                           smem_desc(v_addr + k * 16 * 128, kBlockN * 128), idesc_pv, (n_done[x] > 0 || k > 0) ? 1u : 0u);
+                tc_commit(v_empty + vs);
+                ++n_done[x];
+                return true;
+            };
+            for (int i = 0; i < st.n_tiles && ok; ++i) {
+                const int ks = i % P::kKStages;
+                ok = mbar_wait(k_full + ks, (i / P::kKStages) & 1, abort_flag, status, 7);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t k_addr = smem_u32(smem + P::kK + ks * P::kTileBytes);
+                for (int x = 0; x < 2 && ok; ++x) {
+                    const bool present = (x == 0) || st.has_b;
+                    if (present && st.used_by(x, i)) {
+                        if (pending[x] >= 0) {
+                            const int ip = pending[x];
+                            ok = issue_pv(x, ip);
+                            if (!ok) break;
+                            // a V stage is released by two commits: pay the other tile's share if it skipped ip
+                            if (!(((1 - x) == 0 || st.has_b) && st.used_by(1 - x, ip))) tc_commit(v_empty + ip % P::kVStages);
+                        }
+                        const uint32_t q_addr = smem_u32(smem + P::kQ + x * P::kTileBytes);
+#pragma unroll
+                        for (int k = 0; k < D / 16; ++k) {
+                            const uint32_t off = (k / 4) * (kBlockM * 128) + (k % 4) * 32;
+                            mma_ss(tmem_base + col_s(x), smem_desc(q_addr + off, 0), smem_desc(k_addr + off, 0),
+                                   idesc_qk, k > 0 ? 1u : 0u);
+                        }
+                        tc_commit(s_full + x);
+                        tc_commit(k_empty + ks);
+                        pending[x] = i;
+                    } else {
+                        tc_commit(k_empty + ks);  // the share of a tile that skips this stream tile
+                    }
+                }
+            }
+            for (int x = 0; x < 2 && ok; ++x) {
+                if (pending[x] >= 0) {
+                    const int ip = pending[x];
+                    ok = issue_pv(x, ip);
+                    if (!ok) break;
+                    if (!(((1 - x) == 0 || st.has_b) && st.used_by(1 - x, ip))) tc_commit(v_empty + ip % P::kVStages);
+                    tc_commit(o_final + x);
+                }
+            }
+        }
+    } else if (warp >= 4) {
+        // ------------------------------------------------------------ softmax + epilogue
+        const int x = (warp - 4) >> 2;                 // 0: tile A, 1: tile B
+        const int row_in_tile = ((warp & 3) << 5) | lane;
+        const int t = R0 + x * kBlockM + row_in_tile;  // this thread's query position
+        const bool tile_present = (x == 0) || st.has_b;
+        if (tile_present) {
+            const uint32_t lane_addr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+            const int tq = min(t, N - 1);              // rows past N mimic the last row (never stored)
+            const int c = tq / C;
+            const int lim_sel = c >= 2 ? (c - 1) * lam : 0;
+            const int loc_lo = c >= 1 ? (c - 1) * C : 0;
+            float m_used = -INFINITY, l_sum = 0.f;     // log2 domain
+            int n_seen = 0;
+            bool ok = true;
+            for (int i = 0; i < st.n_tiles && ok; ++i) {
+                if (!st.used_by(x, i)) continue;
+                // visible column interval [lo, hi] of this row in stream tile i
+                int lo, hi;
+                if (st.is_sel(i)) {
+                    lo = 0;
+                    hi = lim_sel - i * kBlockN - 1;
+                } else {
+                    const int p0 = st.loc_m(i) * kBlockN;
+                    lo = loc_lo - p0;
+                    hi = tq - p0;
+                }
+                lo = max(lo, 0);
+                hi = min(hi, kBlockN - 1);
+                const bool need_mask = __any_sync(0xffffffffu, lo > 0 || hi < kBlockN - 1);
+                ok = mbar_wait(s_full + x, n_seen & 1, abort_flag, status, 8);
+                if (!ok) break;
+                tc_fence_after();
+                uint32_t sr[128];
+                tmem_ld32(lane_addr + col_s(x) + 0, sr + 0);
+                tmem_ld32(lane_addr + col_s(x) + 32, sr + 32);
+                tmem_ld32(lane_addr + col_s(x) + 64, sr + 64);
+                tmem_ld32(lane_addr + col_s(x) + 96, sr + 96);
+                tmem_wait_ld();
+                float *s = reinterpret_cast<float *>(sr);
+                if (need_mask) {
+#pragma unroll
+                    for (int j = 0; j < 128; ++j)
+                        if (j < lo || j > hi) s[j] = -INFINITY;
+                }
+                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+                for (int j = 0; j < 128; j += 4) {
+                    mx0 = fmaxf(mx0, s[j]);
+                    mx1 = fmaxf(mx1, s[j + 1]);
+                    mx2 = fmaxf(mx2, s[j + 2]);
+                    mx3 = fmaxf(mx3, s[j + 3]);
+                }
+                const float mt = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * scale_log2;
+                // lazy rescale: keep the old reference unless the new maximum exceeds it by 2^8
+                const bool grow = mt > m_used + 8.f;
+                float alpha = 1.f;
+                if (grow) {
+                    alpha = (m_used == -INFINITY) ? 0.f : ex2(m_used - mt);
+                    m_used = mt;
+                }
+                if (n_seen > 0 && __any_sync(0xffffffffu, grow)) {
+                    // S of this tile was committed after the previous P V product: O is quiescent
+#pragma unroll
+                    for (int q = 0; q < D / 32; ++q) {
+                        uint32_t orow[32];
+                        tmem_ld32(lane_addr + col_o(x) + q * 32, orow);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) orow[j] = __float_as_uint(__uint_as_float(orow[j]) * alpha);
+                        tmem_st32(lane_addr + col_o(x) + q * 32, orow);
+                    }
+                }
+                l_sum *= alpha;
+                const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
+                float acc0 = 0.f, acc1 = 0.f;
+#pragma unroll
+                for (int q = 0; q < 2; ++q) {
+                    uint32_t pk[32];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        float p0 = ex2(fmaf(s[q * 64 + 2 * j], scale_log2, neg_m));
+                        float p1 = ex2(fmaf(s[q * 64 + 2 * j + 1], scale_log2, neg_m));
+                        acc0 += p0;
+                        acc1 += p1;
+                        pk[j] = pack_bf16(p0, p1);
+                    }
+                    tmem_st32(lane_addr + col_s(x) + q * 32, pk);
+                }
+                l_sum += acc0 + acc1;
+                tmem_wait_st();
+                tc_fence_before();
+                mbar_arrive(p_full + x);
+                ++n_seen;
+            }
+            // ---- epilogue: y = (O e^{m-ms} + e^{-ms} N_LA) / (l e^{m-ms} + e^{-ms} D_LA), ms = max(m, 0)
+            if (ok) ok = mbar_wait(o_final + x, 0, abort_flag, status, 9);
+            if (ok) {
+                tc_fence_after();
+                const long long row_off = ((long long)bh * N + t) * D;
+                float fs = 1.f, fl = 0.f, dla = 0.f;
+                if (D_LA != nullptr && t < N) {
+                    dla = D_LA[(long long)bh * N + t];
+                    if (dla > 0.f) {
+                        const float m_nat = m_used * 0.6931471805599453f;
+                        const float ms = fmaxf(m_nat, 0.f);
+                        fs = __expf(m_nat - ms);
+                        fl = __expf(-ms);
+                    }
+                }
+                const float inv = 1.f / (l_sum * fs + fl * dla);
+#pragma unroll
+                for (int q = 0; q < D / 32; ++q) {
+                    uint32_t orow[32];
+                    tmem_ld32(lane_addr + col_o(x) + q * 32, orow);
+                    tmem_wait_ld();
+                    if (t < N) {
+                        uint32_t out[16];
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            float a0 = __uint_as_float(orow[2 * j]) * fs, a1 = __uint_as_float(orow[2 * j + 1]) * fs;
+                            if (dla > 0.f) {
+                                const float2 nl = *reinterpret_cast<const float2 *>(N_LA + row_off + q * 32 + 2 * j);
+                                a0 += fl * nl.x;
+                                a1 += fl * nl.y;
+                            }
+                            out[j] = pack_bf16(a0 * inv, a1 * inv);
+                        }
+                        uint4 *dst = reinterpret_cast<uint4 *>(Y + row_off + q * 32);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) dst[j] = make_uint4(out[4 * j], out[4 * j + 1], out[4 * j + 2], out[4 * j + 3]);
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+// K_sel / V_sel [B*H, sel_rows, d]: row j < n_valid is row sel_idx[j] of the head's K / V
+// (a -1 entry, or a row of the padding, is zero).  One warp per row.
+template <int D>
+__global__ void __launch_bounds__(256)
+compact_kernel(const __nv_bfloat16 *__restrict__ K, const __nv_bfloat16 *__restrict__ V,
+               const int32_t *__restrict__ sel_idx, __nv_bfloat16 *__restrict__ Ksel,
+               __nv_bfloat16 *__restrict__ Vsel, int H, int Hkv, long long N, long long n_idx, long long sel_rows) {
+    const int bh = blockIdx.y, b = bh / H, h = bh % H, kvh = h / (H / Hkv);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long j = (long long)blockIdx.x * 8 + warp;
+    if (j >= sel_rows) return;
+    long long p = -1;
+    if (j < n_idx) p = sel_idx[(long long)bh * n_idx + j];
+    constexpr int kVec = D / 8;  // uint4 per row
+    uint4 kk = make_uint4(0, 0, 0, 0), vv = kk;
+    if (lane < kVec && p >= 0) {
+        kk = reinterpret_cast<const uint4 *>(K + (((long long)b * Hkv + kvh) * N + p) * D)[lane];
+        vv = reinterpret_cast<const uint4 *>(V + (((long long)b * Hkv + kvh) * N + p) * D)[lane];
+    }
+    if (lane < kVec) {
+        reinterpret_cast<uint4 *>(Ksel + ((long long)bh * sel_rows + j) * D)[lane] = kk;
+        reinterpret_cast<uint4 *>(Vsel + ((long long)bh * sel_rows + j) * D)[lane] = vv;
+    }
+}
+
+// ----------------------------------------------------------------- host side
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+// 2-D bf16 tensor [rows, d] tiled in boxes of [128 rows, 64 columns] with 128-byte swizzle.
+bool make_map(CUtensorMap *m, const void *base, unsigned long long rows, int d) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)d * 2};
+    cuuint32_t box[2] = {64, 128};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int D>
+int launch_tc(const still_params_t *p, long long N, const void *Q, const void *K, const void *V,
+              const int32_t *sel_idx, const float *N_LA, const float *D_LA, void *Y, void *k_sel, void *v_sel,
+              long long sel_rows, int *status, cudaStream_t st, int *launches) {
+    using bf = __nv_bfloat16;
+    const long long T = (N + p->chunk - 1) / p->chunk, BH = (long long)p->B * p->H;
+    const long long n_idx = T * p->topk;
+    {
+        dim3 grid((unsigned)((sel_rows + 7) / 8), (unsigned)BH);
+        compact_kernel<D><<<grid, 256, 0, st>>>((const bf *)K, (const bf *)V, sel_idx, (bf *)k_sel, (bf *)v_sel, p->H,
+                                               p->Hkv, N, n_idx, sel_rows);
+        ++*launches;
+        if (cudaGetLastError() != cudaSuccess) return STILL_ERR_CUDA;
+    }
+    CUtensorMap tq, tk, tv, tks, tvs;
+    if (!make_map(&tq, Q, (unsigned long long)BH * N, D) ||
+        !make_map(&tk, K, (unsigned long long)p->B * p->Hkv * N, D) ||
+        !make_map(&tv, V, (unsigned long long)p->B * p->Hkv * N, D) ||
+        !make_map(&tks, k_sel, (unsigned long long)BH * sel_rows, D) ||
+        !make_map(&tvs, v_sel, (unsigned long long)BH * sel_rows, D))
+        return STILL_ERR_CUDA;
+    const int n_qblocks = (int)((N + 2 * kBlockM - 1) / (2 * kBlockM));
+    if (cudaFuncSetAttribute(sa_merge_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             SmemPlan<D>::kAlloc) != cudaSuccess)
+        return STILL_ERR_CUDA;
+    dim3 grid((unsigned)n_qblocks, (unsigned)BH);
+    profile_mark_begin(st);
+    sa_merge_tc_kernel<D><<<grid, kThreads, SmemPlan<D>::kAlloc, st>>>(
+        tq, tk, tv, tks, tvs, N_LA, D_LA, (bf *)Y, status, p->H, p->Hkv, (int)N, p->chunk, p->topk, (int)sel_rows,
+        p->sm_scale * 1.4426950408889634f, n_qblocks);
+    profile_mark_end(st);
+    ++*launches;
+    if (cudaGetLastError() != cudaSuccess) return STILL_ERR_CUDA;
+    return STILL_OK;
+}
+
+}  // namespace
+
+bool tc_supported(const still_params_t *p) {
+    return p->dtype == STILL_DTYPE_BF16 && (p->d == 64 || p->d == 128) && (p->chunk == 64 || p->chunk == 128);
+}
+
+long long tc_sel_rows(const still_params_t *p, long long N) {
+    const long long T = (N + p->chunk - 1) / p->chunk;
+    return (T * p->topk + kBlockN - 1) / kBlockN * kBlockN + kBlockN;
+}
+
+int tc_sa_merge(const still_params_t *p, long long N, const void *Q, const void *K, const void *V,
+                const int32_t *sel_idx, const float *N_LA, const float *D_LA, void *Y, void *k_sel, void *v_sel,
+                long long sel_rows, int *status_words, cudaStream_t st, int *launches) {
+    if ((long long)p->B * p->H * std::max(N, sel_rows) >= (1ll << 31)) return STILL_ERR_UNSUPPORTED;  // TMA row coordinate
+    if (p->d == 64)
+        return launch_tc<64>(p, N, Q, K, V, sel_idx, N_LA, D_LA, Y, k_sel, v_sel, sel_rows, status_words, st, launches);
+    return launch_tc<128>(p, N, Q, K, V, sel_idx, N_LA, D_LA, Y, k_sel, v_sel, sel_rows, status_words, st, launches);
 }
 
 }  // namespace still
