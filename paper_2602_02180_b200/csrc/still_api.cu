@@ -240,7 +240,11 @@ static int fwd_typed(const still_params_t *p, long long N, const T *Q, const T *
     }
 
     // (1)+(2) Self-Saliency Score and per-chunk top-k.
-    if ((rc = launch_score_select<T>(p, N, w.T, Q, K, sc, sel, st)) != STILL_OK) return rc;
+    if (w.tc)
+        rc = tc_score_select(p, N, Q, K, sc, sel, reinterpret_cast<int *>(ws + w.status), st, &g_launches);
+    else
+        rc = launch_score_select<T>(p, N, w.T, Q, K, sc, sel, st);
+    if (rc != STILL_OK) return rc;
 
     // (3) NP-Map + linear-attention scan (skipped when no token can be in M^LA).
     float *nla = nullptr, *dla = nullptr;

@@ -557,6 +557,176 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     }
 }
 
+// ---------------------------------------------------------------------------
+// Self-Saliency Score (Sec. 3.1; Algorithm 1 "Compute Self-Saliency Score") and
+// per-chunk top-k (Sec. 3.3, delayed selection) on tensor cores.
+// One CTA scores 128 consecutive query rows of one (batch, head): one UMMA of
+// shape 128 x 256 x d gives the logits of those rows against the 256 keys at
+// positions [R0-128, R0+128) -- s_prev and s_in of Algorithm 1 side by side.  A
+// thread owns one row; its window is the last C keys up to itself, i.e. the
+// elements j in [lane+1, lane+C] of the C+32 columns its warp reads from TMEM
+// (element lane+C is the token itself).  With e_j = exp(l_j - max), Z = sum e_j,
+// Z' = sum_{j != t} e_j:  a_diag_j = e_j / Z,  a_nodiag_j = e_j / Z' (0 at j = t),
+// Score = sum_j a_diag_j log((a_diag_j + eps) / (a_nodiag_j + eps)).
+// Warps: 0 TMA producer, 1 MMA issuer, 2-5 score (TMEM lane quarter = warp % 4).
+// ---------------------------------------------------------------------------
+template <int D, int C>
+__global__ void __launch_bounds__(192, 2)
+score_select_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                       float *__restrict__ scores, int32_t *__restrict__ sel_idx, int *status, int H, int Hkv,
+                       int N, int lam, float scale_log2, float eps) {
+    constexpr int kQBytes = kBlockM * D * 2, kKBytes = 2 * kBlockN * D * 2;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t *q_s = smem, *k_s = smem + kQBytes;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + kQBytes + kKBytes);  // [0] loads done, [1] logits done
+    uint32_t *tmem_base_slot = reinterpret_cast<uint32_t *>(bars + 2);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_base_slot + 1);
+    float *sc = reinterpret_cast<float *>(tmem_base_slot + 2);                // [128]
+    int *flag = reinterpret_cast<int *>(sc + kBlockM);                         // [128]
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int bh = blockIdx.y, b = bh / H, h = bh % H, kvh = h / (H / Hkv);
+    const int R0 = blockIdx.x * kBlockM;
+    const int Tn = (N + C - 1) / C;
+
+    if (threadIdx.x == 0) {
+        mbar_init(bars, 1);
+        mbar_init(bars + 1, 1);
+        *abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_base_slot, 256);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_base_slot;
+
+    if (warp == 0 && lane == 0) {
+        mbar_expect_tx(bars, kQBytes + kKBytes);
+        const int k_row = (b * Hkv + kvh) * N + R0 - kBlockN;  // may be negative or cross into the previous head: masked by position
+        for (int half = 0; half < D / 64; ++half) {
+            tma_load_2d(q_s + half * (kBlockM * 128), &tm_q, bars, half * 64, bh * N + R0);
+            // K-major operand of 256 rows: per 64-column half, rows 0..255 contiguous
+            tma_load_2d(k_s + half * (2 * kBlockN * 128), &tm_k, bars, half * 64, k_row);
+            tma_load_2d(k_s + half * (2 * kBlockN * 128) + kBlockN * 128, &tm_k, bars, half * 64, k_row + kBlockN);
+        }
+    } else if (warp == 1 && lane == 0) {
+        constexpr uint32_t idesc = make_idesc(kBlockM, 2 * kBlockN, false);
+        if (mbar_wait(bars, 0, abort_flag, status, 20)) {
+            tc_fence_after();
+#pragma unroll
+            for (int k = 0; k < D / 16; ++k) {
+                const uint32_t qa = smem_u32(q_s) + (k / 4) * (kBlockM * 128) + (k % 4) * 32;
+                const uint32_t ka = smem_u32(k_s) + (k / 4) * (2 * kBlockN * 128) + (k % 4) * 32;
+                mma_ss(tmem_base, smem_desc(qa, 0), smem_desc(ka, 0), idesc, k > 0 ? 1u : 0u);
+            }
+            tc_commit(bars + 1);
+        }
+    } else if (warp >= 2) {
+        const int wq = warp & 3;                       // TMEM lane quarter this warp may read
+        const int r = wq * 32 + lane, t = R0 + r;
+        const uint32_t taddr = tmem_base + ((uint32_t)(wq * 32) << 16) + (uint32_t)(wq * 32 + kBlockN - C);
+        constexpr int kChunks = (C + 32) / 32;
+        const bool ok = mbar_wait(bars + 1, 0, abort_flag, status, 21);
+        tc_fence_after();
+        float score = 0.f;
+        if (ok) {
+            // element j of the warp's C+32 columns is the key at position R0 + 32 wq - C + j
+            const int pos0 = R0 + wq * 32 - C;
+            float mx = -INFINITY;
+#pragma unroll 1
+            for (int q = 0; q < kChunks; ++q) {
+                uint32_t v[32];
+                tmem_ld32(taddr + q * 32, v);
+                tmem_wait_ld();
+#pragma unroll
+                for (int jj = 0; jj < 32; ++jj) {
+                    const int j = q * 32 + jj;
+                    const bool valid = (j > lane) && (j <= lane + C) && (pos0 + j >= 0);
+                    if (valid) mx = fmaxf(mx, __uint_as_float(v[jj]));
+                }
+            }
+            const float neg_m = -mx * scale_log2;
+            float z_all = 0.f, z_nd = 0.f;
+#pragma unroll 1
+            for (int q = 0; q < kChunks; ++q) {
+                uint32_t v[32];
+                tmem_ld32(taddr + q * 32, v);
+                tmem_wait_ld();
+#pragma unroll
+                for (int jj = 0; jj < 32; ++jj) {
+                    const int j = q * 32 + jj;
+                    const bool valid = (j > lane) && (j <= lane + C) && (pos0 + j >= 0);
+                    const float e = valid ? ex2(fmaf(__uint_as_float(v[jj]), scale_log2, neg_m)) : 0.f;
+                    z_all += e;
+                    if (j != lane + C) z_nd += e;
+                }
+            }
+            const float inv_all = 1.f / z_all, inv_nd = z_nd > 0.f ? 1.f / z_nd : 0.f;
+#pragma unroll 1
+            for (int q = 0; q < kChunks; ++q) {
+                uint32_t v[32];
+                tmem_ld32(taddr + q * 32, v);
+                tmem_wait_ld();
+#pragma unroll
+                for (int jj = 0; jj < 32; ++jj) {
+                    const int j = q * 32 + jj;
+                    const bool valid = (j > lane) && (j <= lane + C) && (pos0 + j >= 0);
+                    const float e = valid ? ex2(fmaf(__uint_as_float(v[jj]), scale_log2, neg_m)) : 0.f;
+                    const float a = e * inv_all;
+                    const float bb = (j != lane + C) ? e * inv_nd : 0.f;
+                    // a * ln((a + eps) / (bb + eps)); an invalid element has a = 0 and adds nothing
+                    score += a * (__log2f(a + eps) - __log2f(bb + eps));
+                }
+            }
+            score *= 0.6931471805599453f;
+        }
+        sc[r] = score;
+        if (ok && t < N && scores != nullptr) scores[(long long)bh * N + t] = score;
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 256);
+    }
+    if (lam <= 0 || *abort_flag) return;
+    // top-k of each chunk of the tile: rank under (score descending, position ascending), NaN as -inf
+    const int tid = threadIdx.x;
+    int selected = 0, cc = 0, rr = 0, n_c = 0;
+    if (tid < kBlockM) {
+        cc = tid / C;
+        rr = tid - cc * C;
+        const int cbase = R0 + cc * C;
+        n_c = min(C, N - cbase);
+        if (rr < n_c) {
+            float mine = sc[tid];
+            if (isnan(mine)) mine = -INFINITY;
+            int rank = 0;
+            for (int j = 0; j < n_c; ++j) {
+                float o = sc[cc * C + j];
+                if (isnan(o)) o = -INFINITY;
+                rank += (o > mine) || (o == mine && j < rr);
+            }
+            selected = rank < lam;
+        }
+        flag[tid] = selected;
+    }
+    __syncthreads();
+    if (tid < kBlockM && n_c > 0) {
+        int32_t *out = sel_idx + ((long long)bh * Tn + (R0 / C + cc)) * lam;
+        int before = 0;
+        for (int j = 0; j < rr; ++j) before += flag[cc * C + j];
+        if (selected) out[before] = R0 + cc * C + rr;
+        const int n_sel = n_c < lam ? n_c : lam;
+        if (rr >= n_sel && rr < lam) out[rr] = -1;
+    }
+}
+
 // K_sel / V_sel [B*H, sel_rows, d]: row j < n_valid is row sel_idx[j] of the head's K / V
 // (a -1 entry, or a row of the padding, is zero).  One warp per row.
 template <int D>
@@ -649,7 +819,35 @@ int launch_tc(const still_params_t *p, long long N, const void *Q, const void *K
     return STILL_OK;
 }
 
+template <int D, int C>
+int launch_score_tc(const still_params_t *p, long long N, const void *Q, const void *K, float *scores,
+                    int32_t *sel_idx, int *status, cudaStream_t st, int *launches) {
+    CUtensorMap tq, tk;
+    const long long BH = (long long)p->B * p->H;
+    if (!make_map(&tq, Q, (unsigned long long)BH * N, D) ||
+        !make_map(&tk, K, (unsigned long long)p->B * p->Hkv * N, D))
+        return STILL_ERR_CUDA;
+    constexpr int kSmem = kBlockM * D * 2 + 2 * kBlockN * D * 2 + 16 + 16 + 2 * kBlockM * 4 + 1024;
+    if (cudaFuncSetAttribute(score_select_tc_kernel<D, C>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) !=
+        cudaSuccess)
+        return STILL_ERR_CUDA;
+    dim3 grid((unsigned)((N + kBlockM - 1) / kBlockM), (unsigned)BH);
+    score_select_tc_kernel<D, C><<<grid, 192, kSmem, st>>>(tq, tk, scores, sel_idx, status, p->H, p->Hkv, (int)N,
+                                                           p->topk, p->sm_scale * 1.4426950408889634f, p->eps);
+    ++*launches;
+    return cudaGetLastError() == cudaSuccess ? STILL_OK : STILL_ERR_CUDA;
+}
+
 }  // namespace
+
+int tc_score_select(const still_params_t *p, long long N, const void *Q, const void *K, float *scores,
+                    int32_t *sel_idx, int *status_words, cudaStream_t st, int *launches) {
+    if ((long long)p->B * p->H * N >= (1ll << 31)) return STILL_ERR_UNSUPPORTED;
+    if (p->d == 64 && p->chunk == 64) return launch_score_tc<64, 64>(p, N, Q, K, scores, sel_idx, status_words, st, launches);
+    if (p->d == 64 && p->chunk == 128) return launch_score_tc<64, 128>(p, N, Q, K, scores, sel_idx, status_words, st, launches);
+    if (p->d == 128 && p->chunk == 64) return launch_score_tc<128, 64>(p, N, Q, K, scores, sel_idx, status_words, st, launches);
+    return launch_score_tc<128, 128>(p, N, Q, K, scores, sel_idx, status_words, st, launches);
+}
 
 bool tc_supported(const still_params_t *p) {
     return p->dtype == STILL_DTYPE_BF16 && (p->d == 64 || p->d == 128) && (p->chunk == 64 || p->chunk == 128);

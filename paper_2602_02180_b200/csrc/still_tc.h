@@ -18,6 +18,9 @@ void profile_mark_end(cudaStream_t st);
 bool tc_supported(const still_params_t *p);
 // Rows per head of the compacted salient K/V copies (selected rows of all chunks plus tile padding).
 long long tc_sel_rows(const still_params_t *p, long long N);
+// Self-Saliency Score + per-chunk top-k on tensor cores (scores may be NULL).
+int tc_score_select(const still_params_t *p, long long N, const void *Q, const void *K, float *scores,
+                    int32_t *sel_idx, int *status_words, cudaStream_t st, int *launches);
 // Compacts the selected K/V rows and runs the softmax-attention + merge kernel.
 int tc_sa_merge(const still_params_t *p, long long N, const void *Q, const void *K, const void *V,
                 const int32_t *sel_idx, const float *N_LA, const float *D_LA, void *Y, void *k_sel,
