@@ -11,7 +11,7 @@ SOURCES = ["still_api.cu", "still_step.cu", "still_tc.cu"]
 HEADERS = ["still_common.cuh", "still_simt.cuh", "still_tc.h", os.path.join("..", "..", "include", "still.h")]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-    "-Xcompiler", "-fPIC", "-shared",
+    "-Xcompiler", "-fPIC", "-shared", "--threads", "0",
 ]
 
 
@@ -28,7 +28,8 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
     if force or _stale():
         nvcc = os.environ.get("NVCC", "nvcc")
         tmp = LIB_PATH + f".{os.getpid()}.tmp"
-        cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp]
+        extra = os.environ.get("STILL_NVCC_EXTRA", "").split()  # e.g. -DSTILL_EXP2_POLY_PAIRS=2
+        cmd = [nvcc] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp]
         cmd += [os.path.join(CSRC, s) for s in SOURCES]
         subprocess.check_call(cmd)
         os.replace(tmp, LIB_PATH)

@@ -38,6 +38,7 @@
 #include <cuda_bf16.h>
 
 #include <algorithm>
+#include <type_traits>
 
 #include "still_common.cuh"
 
@@ -94,6 +95,13 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
         }
     }
     return true;
+}
+// Bounded wait of the failure path: waits for work already in flight even though the CTA has
+// been flagged as aborted.
+__device__ __forceinline__ void mbar_wait_drain(uint64_t *bar, uint32_t parity) {
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity))
+        if (clock64() - t0 > kWaitLimitCycles) return;
 }
 __device__ __forceinline__ void fence_barrier_init() {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -184,6 +192,45 @@ __device__ __forceinline__ float ex2(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+// Register re-allocation between warpgroups (all four warps of a warpgroup execute it).
+template <uint32_t kRegs>
+__device__ __forceinline__ void reg_inc() {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegs));
+}
+template <uint32_t kRegs>
+__device__ __forceinline__ void reg_dec() {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegs));
+}
+
+// 2^x for a pair of arguments on the FMA pipes (the MUFU unit, 16 ex2 per clock per SM, is as
+// busy as the tensor pipe in this kernel).  Cody-Waite split with the rounding done by the
+// addition of 1.5 * 2^23:  t = s * scale + (magic - m)  has round(x) in its low mantissa bits
+// (x = s * scale - m, m an integer),  f = s * scale - m - round(x)  lies in [-1/2, 1/2],
+// 2^f is a cubic (minimax fit of the relative error, 7.5e-5: well below the bf16 rounding
+// of P), and round(x) is added to the exponent field.  Requires x >= -126, which the caller
+// guarantees by clamping s from below.
+__device__ __forceinline__ float2 exp2_poly2(float2 sv, float2 scale2, float2 k2) {
+    const float2 t = __ffma2_rn(sv, scale2, k2);
+    const float2 c = __ffma2_rn(t, make_float2(-1.f, -1.f), k2);   // -(m + round(x))
+    const float2 f = __ffma2_rn(sv, scale2, c);
+    float2 p = __ffma2_rn(f, make_float2(0.0551716685f, 0.0551716685f), make_float2(0.24261114f, 0.24261114f));
+    p = __ffma2_rn(p, f, make_float2(0.693260968f, 0.693260968f));
+    p = __ffma2_rn(p, f, make_float2(0.999928057f, 0.999928057f));
+    float2 r;
+    r.x = __int_as_float(__float_as_int(p.x) + (__float_as_int(t.x) << 23));
+    r.y = __int_as_float(__float_as_int(p.y) + (__float_as_int(t.y) << 23));
+    return r;
+}
+// Of every four column pairs of a softmax row, this many take the polynomial instead of MUFU.
+#ifndef STILL_EXP2_POLY_PAIRS
+#define STILL_EXP2_POLY_PAIRS 0
+#endif
+
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     uint32_t r;
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
@@ -219,7 +266,7 @@ struct SmemPlan {
     static constexpr int kK = kQ + 2 * kTileBytes;
     static constexpr int kV = kK + kKStages * kTileBytes;
     static constexpr int kBar = kV + kVStages * kTileBytes;    // mbarriers
-    static constexpr int kNumBars = 1 + 2 * kKStages + 2 * kVStages + 6;
+    static constexpr int kNumBars = 1 + 2 * kKStages + 2 * kVStages + 9;
     static constexpr int kMisc = kBar + kNumBars * 8;          // tmem base, abort flag
     static constexpr int kTotal = kMisc + 16;
     static constexpr int kAlloc = kTotal + 1024;               // slack to align the base to 1024
@@ -262,8 +309,9 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     uint64_t *k_full = bars + 1, *k_empty = k_full + P::kKStages;
     uint64_t *v_full = k_empty + P::kKStages, *v_empty = v_full + P::kVStages;
     uint64_t *s_full = v_empty + P::kVStages;  // [2]
-    uint64_t *p_full = s_full + 2;             // [2]
-    uint64_t *o_final = p_full + 2;            // [2]
+    uint64_t *p_half = s_full + 2;             // [2][2]: columns [0,64) / [64,128) of P_X are in TMEM
+    uint64_t *o_final = p_half + 4;            // [2]
+    uint64_t *drain = o_final + 2;             // MMA warp: everything issued has completed (failure path)
     uint32_t *tmem_base_slot = reinterpret_cast<uint32_t *>(smem + P::kMisc);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + P::kMisc + 8);
 
@@ -292,7 +340,9 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         mbar_init(q_full, 1);
         for (int i = 0; i < P::kKStages; ++i) { mbar_init(k_full + i, 1); mbar_init(k_empty + i, 2); }
         for (int i = 0; i < P::kVStages; ++i) { mbar_init(v_full + i, 1); mbar_init(v_empty + i, 2); }
-        for (int i = 0; i < 2; ++i) { mbar_init(s_full + i, 1); mbar_init(p_full + i, 128); mbar_init(o_final + i, 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(s_full + i, 1); mbar_init(o_final + i, 1); }
+        for (int i = 0; i < 4; ++i) mbar_init(p_half + i, 128);
+        mbar_init(drain, 1);
         *abort_flag = 0;
         fence_barrier_init();
     }
@@ -308,6 +358,10 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     auto col_s = [](int x) -> uint32_t { return (uint32_t)x * 128u; };
     auto col_o = [](int x) -> uint32_t { return 256u + (uint32_t)x * (uint32_t)D; };
 
+    // The softmax threads keep a whole 128-column row in registers: move registers from the
+    // load / MMA warpgroup to the two softmax warpgroups (128 * 64 + 256 * 216 <= 384 * 168).
+    if (warp < 4) {
+    reg_dec<64>();
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
@@ -317,35 +371,60 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 for (int half = 0; half < D / 64; ++half)
                     tma_load_2d(smem + P::kQ + x * P::kTileBytes + half * (kBlockM * 128), &tm_q, q_full, half * 64,
                                 q_row + x * kBlockM);
+            // K and V rings advance independently, each as far ahead as its free stages allow.
             bool ok = true;
-            int armed_k = 0, armed_v = 0;
-            for (int i = 0; i < st.n_tiles && ok; ++i) {
-                const bool sel = st.is_sel(i);
-                const CUtensorMap *mk = sel ? &tm_ksel : &tm_k, *mv = sel ? &tm_vsel : &tm_v;
-                const int row = sel ? bh * sel_rows + i * kBlockN : (b * Hkv + kvh) * N + st.loc_m(i) * kBlockN;
-                const int ks = i % P::kKStages, vs = i % P::kVStages;
-                ok = mbar_wait(k_empty + ks, ((i / P::kKStages) & 1) ^ 1, abort_flag, status, 1);
-                if (!ok) break;
-                mbar_expect_tx(k_full + ks, P::kTileBytes);
-                for (int half = 0; half < D / 64; ++half)
-                    tma_load_2d(smem + P::kK + ks * P::kTileBytes + half * (kBlockN * 128), mk, k_full + ks, half * 64, row);
-                armed_k = i + 1;
-                ok = mbar_wait(v_empty + vs, ((i / P::kVStages) & 1) ^ 1, abort_flag, status, 2);
-                if (!ok) break;
-                mbar_expect_tx(v_full + vs, P::kTileBytes);
-                for (int half = 0; half < D / 64; ++half)
-                    tma_load_2d(smem + P::kV + vs * P::kTileBytes + half * (kBlockN * 128), mv, v_full + vs, half * 64, row);
-                armed_v = i + 1;
+            int armed_k = 0, armed_v = 0, spins = 0;
+            long long t0 = clock64();
+            while (armed_k < st.n_tiles || armed_v < st.n_tiles) {
+                bool progressed = false;
+                if (armed_k < st.n_tiles) {
+                    const int i = armed_k, ks = i % P::kKStages;
+                    if (mbar_try_wait(k_empty + ks, ((i / P::kKStages) & 1) ^ 1)) {
+                        const bool sel = st.is_sel(i);
+                        const int row = sel ? bh * sel_rows + i * kBlockN : (b * Hkv + kvh) * N + st.loc_m(i) * kBlockN;
+                        mbar_expect_tx(k_full + ks, P::kTileBytes);
+                        for (int half = 0; half < D / 64; ++half)
+                            tma_load_2d(smem + P::kK + ks * P::kTileBytes + half * (kBlockN * 128), sel ? &tm_ksel : &tm_k,
+                                        k_full + ks, half * 64, row);
+                        ++armed_k;
+                        progressed = true;
+                    }
+                }
+                if (armed_v < st.n_tiles) {
+                    const int i = armed_v, vs = i % P::kVStages;
+                    if (mbar_try_wait(v_empty + vs, ((i / P::kVStages) & 1) ^ 1)) {
+                        const bool sel = st.is_sel(i);
+                        const int row = sel ? bh * sel_rows + i * kBlockN : (b * Hkv + kvh) * N + st.loc_m(i) * kBlockN;
+                        mbar_expect_tx(v_full + vs, P::kTileBytes);
+                        for (int half = 0; half < D / 64; ++half)
+                            tma_load_2d(smem + P::kV + vs * P::kTileBytes + half * (kBlockN * 128), sel ? &tm_vsel : &tm_v,
+                                        v_full + vs, half * 64, row);
+                        ++armed_v;
+                        progressed = true;
+                    }
+                }
+                if (progressed) {
+                    spins = 0;
+                } else if ((++spins & 1023) == 0) {
+                    if (spins == 1024) t0 = clock64();
+                    if (*abort_flag) { ok = false; break; }
+                    if (clock64() - t0 > kWaitLimitCycles) {
+                        *abort_flag = 1;
+                        report_status(status, STILL_ERR_DEVICE_TIMEOUT, 1);
+                        ok = false;
+                        break;
+                    }
+                }
             }
             if (!ok) {
                 // leave no copy in flight behind: wait (bounded) for the loads already issued
                 if (armed_k > 0) {
                     int i = armed_k - 1;
-                    mbar_wait(k_full + i % P::kKStages, (i / P::kKStages) & 1, abort_flag, status, 3);
+                    mbar_wait_drain(k_full + i % P::kKStages, (i / P::kKStages) & 1);
                 }
                 if (armed_v > 0) {
                     int i = armed_v - 1;
-                    mbar_wait(v_full + i % P::kVStages, (i / P::kVStages) & 1, abort_flag, status, 3);
+                    mbar_wait_drain(v_full + i % P::kVStages, (i / P::kVStages) & 1);
                 }
             }
         }
@@ -359,15 +438,21 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             int pending[2] = {-1, -1};   // stream tile whose P V product is still to be issued
             int n_done[2] = {0, 0};      // tiles processed per query tile (phase of p_full)
             auto issue_pv = [&](int x, int ip) -> bool {
-                if (!mbar_wait(p_full + x, n_done[x] & 1, abort_flag, status, 5)) return false;
                 const int vs = ip % P::kVStages;
+                if (!mbar_wait(p_half + 2 * x, n_done[x] & 1, abort_flag, status, 5)) return false;
                 if (!mbar_wait(v_full + vs, (ip / P::kVStages) & 1, abort_flag, status, 6)) return false;
                 tc_fence_after();
                 const uint32_t v_addr = smem_u32(smem + P::kV + vs * P::kTileBytes);
 #pragma unroll
-                for (int k = 0; k < kBlockN / 16; ++k)
+                for (int k = 0; k < kBlockN / 32; ++k)
                     mma_ts(tmem_base + col_o(x), tmem_base + col_s(x) + k * 8,
                            smem_desc(v_addr + k * 16 * 128, kBlockN * 128), idesc_pv, (n_done[x] > 0 || k > 0) ? 1u : 0u);
+                if (!mbar_wait(p_half + 2 * x + 1, n_done[x] & 1, abort_flag, status, 5)) return false;
+                tc_fence_after();
+#pragma unroll
+                for (int k = kBlockN / 32; k < kBlockN / 16; ++k)
+                    mma_ts(tmem_base + col_o(x), tmem_base + col_s(x) + k * 8,
+                           smem_desc(v_addr + k * 16 * 128, kBlockN * 128), idesc_pv, 1u);
                 tc_commit(v_empty + vs);
                 ++n_done[x];
                 return true;
@@ -412,8 +497,14 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     tc_commit(o_final + x);
                 }
             }
+            if (!ok) {  // no MMA may still be running when tensor memory is freed
+                tc_commit(drain);
+                mbar_wait_drain(drain, 0);
+            }
         }
-    } else if (warp >= 4) {
+    }
+    } else {
+        reg_inc<216>();
         // ------------------------------------------------------------ softmax + epilogue
         const int x = (warp - 4) >> 2;                 // 0: tile A, 1: tile B
         const int row_in_tile = ((warp & 3) << 5) | lane;
@@ -426,6 +517,7 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             const int lim_sel = c >= 2 ? (c - 1) * lam : 0;
             const int loc_lo = c >= 1 ? (c - 1) * C : 0;
             float m_used = -INFINITY, l_sum = 0.f;     // log2 domain
+            const float inv_scale_log2 = 1.f / scale_log2;
             int n_seen = 0;
             bool ok = true;
             for (int i = 0; i < st.n_tiles && ok; ++i) {
@@ -460,19 +552,22 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 }
                 float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-                for (int j = 0; j < 128; j += 4) {
-                    mx0 = fmaxf(mx0, s[j]);
-                    mx1 = fmaxf(mx1, s[j + 1]);
-                    mx2 = fmaxf(mx2, s[j + 2]);
-                    mx3 = fmaxf(mx3, s[j + 3]);
+                for (int j = 0; j < 128; j += 8) {
+                    mx0 = max3(mx0, s[j], s[j + 1]);
+                    mx1 = max3(mx1, s[j + 2], s[j + 3]);
+                    mx2 = max3(mx2, s[j + 4], s[j + 5]);
+                    mx3 = max3(mx3, s[j + 6], s[j + 7]);
                 }
                 const float mt = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * scale_log2;
-                // lazy rescale: keep the old reference unless the new maximum exceeds it by 2^8
+                // lazy rescale: keep the old reference unless the new maximum exceeds it by 2^8.  The
+                // reference is an integer (any reference within range is valid), which lets the
+                // polynomial 2^x take its integer part straight from the mantissa of one FMA.
                 const bool grow = mt > m_used + 8.f;
                 float alpha = 1.f;
                 if (grow) {
-                    alpha = (m_used == -INFINITY) ? 0.f : ex2(m_used - mt);
-                    m_used = mt;
+                    const float m_new = ceilf(mt);
+                    alpha = (m_used == -INFINITY) ? 0.f : ex2(m_used - m_new);
+                    m_used = m_new;
                 }
                 if (n_seen > 0 && __any_sync(0xffffffffu, grow)) {
                     // S of this tile was committed after the previous P V product: O is quiescent
@@ -488,24 +583,51 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 }
                 l_sum *= alpha;
                 const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
-                float acc0 = 0.f, acc1 = 0.f;
+                const float2 scale2 = make_float2(scale_log2, scale_log2), negm2 = make_float2(neg_m, neg_m);
+                // polynomial path: unmasked tiles with a reference of moderate size (uniform per warp)
+                const bool poly = STILL_EXP2_POLY_PAIRS > 0 && !need_mask &&
+                                  __all_sync(0xffffffffu, fabsf(m_used) < 1048576.f);
+                const float k_magic = 12582912.f + neg_m;                 // 1.5 * 2^23 - m
+                const float s_floor = (m_used - 125.f) * inv_scale_log2;  // keeps x >= -126
+                const float2 k2 = make_float2(k_magic, k_magic);
+                float2 acc = make_float2(0.f, 0.f);
+                // P = 2^(s * scale - m) as bf16 over S, in two halves of 64 columns; the MMA warp
+                // starts on the first half while the second is computed.
+                auto exp_row = [&](auto poly_pairs) {
+                    constexpr int kPoly = decltype(poly_pairs)::value;
 #pragma unroll
-                for (int q = 0; q < 2; ++q) {
-                    uint32_t pk[32];
+                    for (int q = 0; q < 2; ++q) {
+                        uint32_t pk[32];
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        float p0 = ex2(fmaf(s[q * 64 + 2 * j], scale_log2, neg_m));
-                        float p1 = ex2(fmaf(s[q * 64 + 2 * j + 1], scale_log2, neg_m));
-                        acc0 += p0;
-                        acc1 += p1;
-                        pk[j] = pack_bf16(p0, p1);
+                        for (int j = 0; j < 32; ++j) {
+                            float2 sv = make_float2(s[q * 64 + 2 * j], s[q * 64 + 2 * j + 1]);
+                            float2 pr;
+                            if ((j & 3) < kPoly) {
+                                sv.x = fmaxf(sv.x, s_floor);
+                                sv.y = fmaxf(sv.y, s_floor);
+                                pr = exp2_poly2(sv, scale2, k2);
+                            } else {
+                                const float2 xv = __ffma2_rn(sv, scale2, negm2);
+                                pr = make_float2(ex2(xv.x), ex2(xv.y));
+                            }
+                            acc = __fadd2_rn(acc, pr);
+                            pk[j] = pack_bf16(pr.x, pr.y);
+                            if (q == 1 && j == 12) {
+                                // the first half of P has had time to land: hand it to the MMA warp
+                                tmem_wait_st();
+                                tc_fence_before();
+                                mbar_arrive(p_half + 2 * x);
+                            }
+                        }
+                        tmem_st32(lane_addr + col_s(x) + q * 32, pk);
                     }
-                    tmem_st32(lane_addr + col_s(x) + q * 32, pk);
-                }
-                l_sum += acc0 + acc1;
+                };
+                if (poly) exp_row(std::integral_constant<int, STILL_EXP2_POLY_PAIRS>{});
+                else exp_row(std::integral_constant<int, 0>{});
+                l_sum += acc.x + acc.y;
                 tmem_wait_st();
                 tc_fence_before();
-                mbar_arrive(p_full + x);
+                mbar_arrive(p_half + 2 * x + 1);
                 ++n_seen;
             }
             // ---- epilogue: y = (O e^{m-ms} + e^{-ms} N_LA) / (l e^{m-ms} + e^{-ms} D_LA), ms = max(m, 0)
