@@ -185,6 +185,39 @@ int still_hybrid_attn_fwd_host(const still_params_t *p, int64_t N, const void *h
                                void *cuda_stream);
 
 /*
+ * Prefill without a caller-provided workspace.  (The paper has no counterpart: this is a
+ * packaging variant of still_hybrid_attn_fwd, for callers that cannot allocate device memory --
+ * code that runs inside another runtime's fixed memory plan, a serving loop whose memory was
+ * budgeted at start-up, a context where cudaMalloc is not allowed or would stall the device.)
+ *
+ * The intermediate results that still_hybrid_attn_fwd keeps in `workspace` live instead in a
+ * fixed array of STILL_STATIC_WORKSPACE_BYTES inside the library's device image.  Every GPU on
+ * which the library is used holds that array until the process exits.  The call itself allocates
+ * and frees nothing: no cudaMalloc, no cudaFree, no allocating library routine.
+ *
+ *   - Arguments are those of still_hybrid_attn_fwd without state_out, workspace and their sizes;
+ *     Q, K, V, (G, Wq, bq, Wk, bk), Y, scores, sel_idx are still the caller's device buffers.
+ *   - Limit: still_workspace_bytes(p, N) must not exceed STILL_STATIC_WORKSPACE_BYTES, otherwise
+ *     the call returns STILL_ERR_WORKSPACE_TOO_SMALL and launches nothing.  (With the default
+ *     d_f = d = 64, bf16, B = 1, H = 4 and topk = chunk / 4 this admits N up to about 5000.)
+ *   - The first call on each device looks up the array's device address (one
+ *     cudaGetSymbolAddress, with that device current); make that first call outside any stream
+ *     capture.
+ *   - All calls share the one array, and it keeps whatever the previous call left there.  The
+ *     parts that must start at zero are cleared by every call on its own stream.  Two calls
+ *     that overlap on the GPU (different streams, or different host threads without ordering
+ *     between their streams) race on it: keep calls on one device ordered one after the other.
+ *   - The device status word of the call is not reachable through still_device_status.
+ * Errors: those of still_hybrid_attn_fwd, STILL_ERR_WORKSPACE_TOO_SMALL as above, STILL_ERR_CUDA
+ * if the address look-up fails.
+ */
+#define STILL_STATIC_WORKSPACE_BYTES (16u << 20)
+int still_hybrid_attn_fwd_static(const still_params_t *p, int64_t N, const void *Q, const void *K,
+                                 const void *V, const void *G, const void *Wq, const void *bq,
+                                 const void *Wk, const void *bk, void *Y, float *scores,
+                                 int32_t *sel_idx, void *cuda_stream);
+
+/*
  * Reads the device status word of a workspace (prefill) or of a decode state
  * after synchronising `cuda_stream`.  *status receives STILL_OK or
  * STILL_ERR_DEVICE_TIMEOUT / STILL_ERR_STATE_MISMATCH; *detail (optional)

@@ -6,6 +6,7 @@ from .binding import (  # noqa: F401
     host_arena_bytes,
     hybrid_attn_fwd,
     hybrid_attn_fwd_host,
+    hybrid_attn_fwd_static,
     hybrid_attn_step,
     last_launch_count,
     profile_collect,

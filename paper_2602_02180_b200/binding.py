@@ -91,6 +91,8 @@ def lib():
         L.still_host_arena_bytes.argtypes = [pp, i64]
         L.still_hybrid_attn_fwd_host.restype = ctypes.c_int
         L.still_hybrid_attn_fwd_host.argtypes = [pp, i64] + [vp] * 11 + [vp, sz, vp]
+        L.still_hybrid_attn_fwd_static.restype = ctypes.c_int
+        L.still_hybrid_attn_fwd_static.argtypes = [pp, i64] + [vp] * 11 + [vp]
         L.still_device_status.restype = ctypes.c_int
         L.still_device_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_int)]
         L.still_last_launch_count.restype = ctypes.c_int
@@ -173,6 +175,26 @@ def hybrid_attn_fwd(p: StillParams, Q, K, V, Wq=None, Wk=None, G=None, bq=None, 
     if rc != STILL_OK:
         raise StillError(rc, "still_hybrid_attn_fwd")
     return Y, scores, sel_idx[..., : p.topk]
+
+
+STATIC_WORKSPACE_BYTES = 16 << 20
+
+
+def hybrid_attn_fwd_static(p: StillParams, Q, K, V, Wq=None, Wk=None, G=None, bq=None, bk=None, *, Y, scores,
+                           sel_idx):
+    """still_hybrid_attn_fwd_static: the prefill with its workspace inside the library (for callers
+    that cannot allocate device memory).  Every output buffer is passed in; this wrapper allocates
+    nothing either.  Returns (Y, scores, sel_idx)."""
+    if not Q.is_cuda:
+        raise RuntimeError("still_hybrid_attn_fwd_static needs CUDA tensors; there is no CPU path")
+    c = p.c()
+    rc = lib().still_hybrid_attn_fwd_static(
+        ctypes.byref(c), Q.shape[2], _ptr(Q), _ptr(K), _ptr(V), _ptr(G), _ptr(Wq), _ptr(bq), _ptr(Wk), _ptr(bk),
+        _ptr(Y), _ptr(scores), _ptr(sel_idx), _stream(),
+    )
+    if rc != STILL_OK:
+        raise StillError(rc, "still_hybrid_attn_fwd_static")
+    return Y, scores, sel_idx
 
 
 def hybrid_attn_step(p: StillParams, state, state_max_tokens, t_pos, q, k, v, Wq=None, Wk=None, g=None,

@@ -7,7 +7,7 @@ import subprocess
 _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB_PATH = os.path.join(_HERE, "libstill.so")
-SOURCES = ["still_api.cu", "still_step.cu", "still_tc.cu"]
+SOURCES = ["still_api.cu", "still_step.cu", "still_tc.cu", "still_static.cu"]
 HEADERS = ["still_common.cuh", "still_simt.cuh", "still_tc.h", os.path.join("..", "..", "include", "still.h")]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
