@@ -99,6 +99,34 @@ def test_c2_sampled():
     U.check_outputs(w4, r["Q"], r["K"], r["V"], r["Wq"], r["Wk"], r["Y"], r["scores"], r["sel"], heads, rows=rows)
 
 
+@pytest.mark.parametrize("name,n_heads,n_rows", [("c3", 3, 40), ("c4", 2, 24)])
+def test_full_size_workloads_sampled(name, n_heads, n_rows):
+    # The benchmark's own shapes and launch configuration; the oracle checks sampled heads and rows
+    # (all O(N) steps -- scores, selection -- in full for those heads).
+    w = synth.WORKLOADS[name]
+    r = U.run_prefill(w)
+    assert still.device_status is not None
+    heads = U.sample_heads(w, n_heads, seed=3)
+    rows = U.sample_rows(w.N, n_rows, w.C, seed=3)
+    U.check_selection(r["scores"], r["sel"], w.C, w.k, heads)
+    worst, serr = U.check_outputs(w, r["Q"], r["K"], r["V"], r["Wq"], r["Wk"], r["Y"], r["scores"], r["sel"],
+                                  heads, rows=rows)
+    assert serr < 2e-3
+    print(f"{name} max-abs {worst:.2e} score err {serr:.2e}")
+
+
+def test_c3_companion_quarter_selection_sampled():
+    # lambda = C / 4 at the 32K shape: selection, NP-Map, state scan and merge at scale
+    w = synth.WORKLOADS["c3"].with_(B=1, k=16)
+    r = U.run_prefill(w)
+    heads = U.sample_heads(w, 2, seed=4)
+    rows = U.sample_rows(w.N, 32, w.C, seed=4)
+    U.check_selection(r["scores"], r["sel"], w.C, w.k, heads)
+    worst, serr = U.check_outputs(w, r["Q"], r["K"], r["V"], r["Wq"], r["Wk"], r["Y"], r["scores"], r["sel"],
+                                  heads, rows=rows)
+    print(f"c3 k16 max-abs {worst:.2e} score err {serr:.2e}")
+
+
 def test_invalid_arguments_are_rejected():
     w = _small("t", "bf16", 1, 2, 2, 64, 128, 64, 16)
     Q, K, V = synth.make_qkv(w, "cuda")
