@@ -54,7 +54,7 @@ static inline bool la_active(const still_params_t *p) { return p->topk < p->chun
 struct FwdPlan {
     size_t status, scores, sel_idx, phiQ, phiK, nla, dla, ksel, vsel, total;
     long long T, sel_rows;  // chunks; rows of the compacted salient K/V per head
-    bool la, tc;
+    bool la, tc, tc_la;
 };
 
 static FwdPlan plan_fwd(const still_params_t *p, long long N) {
@@ -65,6 +65,7 @@ static FwdPlan plan_fwd(const still_params_t *p, long long N) {
     w.T = T;
     w.la = la_active(p);
     w.tc = tc_supported(p);
+    w.tc_la = w.la && tc_la_supported(p);
     size_t off = 0;
     auto take = [&](size_t bytes) {
         size_t o = off;
@@ -75,7 +76,7 @@ static FwdPlan plan_fwd(const still_params_t *p, long long N) {
     w.scores = take(BH * (size_t)N * 4);
     w.sel_idx = take(BH * (size_t)T * (size_t)std::max(p->topk, 1) * 4);
     if (w.la) {
-        w.phiQ = take(BH * (size_t)N * dp * es);
+        w.phiQ = take(BH * (size_t)N * dp * (w.tc_la ? 4 : es));  // fp32 features for the TF32 read-out GEMM
         w.phiK = take(BHkv * (size_t)N * dp * es);
         w.nla = take(BH * (size_t)N * p->d * 4);
         w.dla = take(BH * (size_t)N * 4);
@@ -255,10 +256,16 @@ static int fwd_typed(const still_params_t *p, long long N, const T *Q, const T *
         T *phiQ = reinterpret_cast<T *>(ws + w.phiQ), *phiK = reinterpret_cast<T *>(ws + w.phiK);
         nla = reinterpret_cast<float *>(ws + w.nla);
         dla = reinterpret_cast<float *>(ws + w.dla);
-        if ((rc = launch_npmap<T>(p, N, p->H, Q, Wq, bq, phiQ, st)) != STILL_OK) return rc;
-        if ((rc = launch_npmap<T>(p, N, p->Hkv, K, Wk, bk, phiK, st)) != STILL_OK) return rc;
-        if ((rc = launch_la_scan<T>(p, N, w.T, phiQ, phiK, V, G, sel, nla, dla, S_out, z_out, st)) != STILL_OK)
-            return rc;
+        if (w.tc_la) {
+            rc = tc_la_branch(p, N, Q, K, V, G, Wq, bq, Wk, bk, sel, phiQ, phiK, nla, dla, S_out, z_out,
+                              reinterpret_cast<int *>(ws + w.status), st, &g_launches);
+            if (rc != STILL_OK) return rc;
+        } else {
+            if ((rc = launch_npmap<T>(p, N, p->H, Q, Wq, bq, phiQ, st)) != STILL_OK) return rc;
+            if ((rc = launch_npmap<T>(p, N, p->Hkv, K, Wk, bk, phiK, st)) != STILL_OK) return rc;
+            if ((rc = launch_la_scan<T>(p, N, w.T, phiQ, phiK, V, G, sel, nla, dla, S_out, z_out, st)) != STILL_OK)
+                return rc;
+        }
     } else if (state) {
         STILL_CUDA(cudaMemsetAsync(state + L.S, 0, L.scratch - L.S, st));
     }

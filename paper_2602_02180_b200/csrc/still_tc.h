@@ -26,6 +26,17 @@ int tc_sa_merge(const still_params_t *p, long long N, const void *Q, const void 
                 const int32_t *sel_idx, const float *N_LA, const float *D_LA, void *Y, void *k_sel,
                 void *v_sel, long long sel_rows, int *status_words, cudaStream_t st, int *launches);
 
+// ---- tensor-core linear-attention branch of the prefill, bf16 only --------------------
+// True when NP-Map and the chunk-wise state scan of these parameters run on the tcgen05 kernels.
+bool tc_la_supported(const still_params_t *p);
+// NP-Map of Q (fp32 features into phiQ [B,H,N,2 d_f]) and of K (bf16 features into phiK
+// [B,Hkv,N,2 d_f]), then the state scan: N_LA [B,H,N,d] (gated), D_LA [B,H,N]; S_out / z_out
+// (optional) receive the state after the chunks that have left the local region.
+int tc_la_branch(const still_params_t *p, long long N, const void *Q, const void *K, const void *V, const void *G,
+                 const void *Wq, const void *bq, const void *Wk, const void *bk, const int32_t *sel_idx, void *phiQ,
+                 void *phiK, float *nla, float *dla, float *S_out, float *z_out, int *status_words, cudaStream_t st,
+                 int *launches);
+
 // ---- decode step ----------------------------------------------------------------------
 size_t step_scratch_bytes(const still_params_t *p, long long capacity);
 int step_launch(const still_params_t *p, char *state, const still_state_layout_t *L, long long t_pos,
