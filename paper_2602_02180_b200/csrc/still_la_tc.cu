@@ -205,7 +205,7 @@ struct ScanPlan {
     static constexpr int kQ = kU + 2 * kUStage;        // two read-out stages
     static constexpr int kOnes = kQ + 2 * kPhiQ;       // second M atom of the update's A operand
     static constexpr int kBar = kOnes + 64 * 128;
-    static constexpr int kNumBars = 2 + 2 + 2 + 2 + 2 + 3;  // u_full, u_empty, u_masked, q_full, q_empty, r_done, out_free, fin
+    static constexpr int kNumBars = 2 + 2 + 2 + 2 + 2 + 5;  // u_full, u_empty, u_masked, q_full, q_empty, r_done[2], out_free[2], fin
     static constexpr int kMisc = kBar + kNumBars * 8;
     static constexpr int kTotal = kMisc + 16;
 };
@@ -221,7 +221,7 @@ la_scan_tc_kernel(const __grid_constant__ CUtensorMap tm_phik, const __grid_cons
     extern __shared__ __align__(1024) uint8_t smem[];
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + P::kBar);
     uint64_t *u_full = bars, *u_empty = bars + 2, *u_masked = bars + 4, *q_full = bars + 6, *q_empty = bars + 8;
-    uint64_t *r_done = bars + 10, *out_free = bars + 11, *fin = bars + 12;
+    uint64_t *r_done = bars + 10, *out_free = bars + 12, *fin = bars + 14;
     uint32_t *tmem_base_slot = reinterpret_cast<uint32_t *>(smem + P::kMisc);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + P::kMisc + 8);
 
@@ -250,8 +250,10 @@ la_scan_tc_kernel(const __grid_constant__ CUtensorMap tm_phik, const __grid_cons
             mbar_init(q_full + i, 1);
             mbar_init(q_empty + i, 4);
         }
-        mbar_init(r_done, 1);
-        mbar_init(out_free, 4);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(r_done + i, 1);
+            mbar_init(out_free + i, 4);
+        }
         mbar_init(fin, 1);
         *abort_flag = 0;
         fence_barrier_init();
@@ -274,7 +276,8 @@ la_scan_tc_kernel(const __grid_constant__ CUtensorMap tm_phik, const __grid_cons
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_base_slot;
-    const uint32_t col_state = 0, col_out = NF;   // S^T [128 x NF] fp32; read-out result [128 x 64] fp32
+    const uint32_t col_state = 0, col_out = NF;   // S^T [128 x NF] fp32; two read-out results [128 x 64] fp32, so that
+                                                  // the epilogue of one sub-chunk overlaps the MMAs of the next
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
@@ -345,15 +348,15 @@ la_scan_tc_kernel(const __grid_constant__ CUtensorMap tm_phik, const __grid_cons
                     if (!ok) break;
                 }
                 ok = mbar_wait(q_full + (nq & 1), (nq >> 1) & 1, abort_flag, status, 42);
-                if (ok) ok = mbar_wait(out_free, (nq & 1) ^ 1, abort_flag, status, 43);
+                if (ok) ok = mbar_wait(out_free + (nq & 1), ((nq >> 1) & 1) ^ 1, abort_flag, status, 43);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t qs = smem_u32(smem + P::kQ + (nq & 1) * P::kPhiQ);
 #pragma unroll
                 for (int k = 0; k < NF / 8; ++k)   // 8 features per step: 32 bytes within a 32-feature atom
-                    mma_ts_tf32(tmem_base + col_out, tmem_base + col_state + k * 8,
+                    mma_ts_tf32(tmem_base + col_out + (nq & 1) * 64, tmem_base + col_state + k * 8,
                                 smem_desc(qs + (k / 4) * (64 * 128) + (k % 4) * 32, 0), idesc_rd, k > 0 ? 1u : 0u);
-                tc_commit(r_done);
+                tc_commit(r_done + (nq & 1));
                 ++nq;
             }
             // state after the last update (chunks 0 .. Tn-3), for the decode state
@@ -406,13 +409,13 @@ la_scan_tc_kernel(const __grid_constant__ CUtensorMap tm_phik, const __grid_cons
         for (int u = u_first; u < NU; ++u) {
             if ((u + 1) % sc == 0)                                     // tiles of the next chunk's update
                 for (int j = 0; j < sc && nu < n_upd; ++j) mask_tile();
-            if (ok) ok = mbar_wait(r_done, nq & 1, abort_flag, status, 45);
+            if (ok) ok = mbar_wait(r_done + (nq & 1), (nq >> 1) & 1, abort_flag, status, 45);
             ok = __all_sync(0xffffffffu, ok);
             if (ok) {
                 tc_fence_after();
                 uint32_t o[64];
-                tmem_ld32(taddr + col_out, o);
-                tmem_ld32(taddr + col_out + 32, o + 32);
+                tmem_ld32(taddr + col_out + (nq & 1) * 64, o);
+                tmem_ld32(taddr + col_out + (nq & 1) * 64 + 32, o + 32);
                 tmem_wait_ld();
                 const int base = u * 64;
                 if (e < 64) {
@@ -433,7 +436,7 @@ la_scan_tc_kernel(const __grid_constant__ CUtensorMap tm_phik, const __grid_cons
             }
             __syncwarp();
             if (lane == 0) {
-                mbar_arrive(out_free);
+                mbar_arrive(out_free + (nq & 1));
                 mbar_arrive(q_empty + (nq & 1));
             }
             ++nq;
