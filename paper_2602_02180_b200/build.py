@@ -8,7 +8,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB_PATH = os.path.join(_HERE, "libstill.so")
 SOURCES = ["still_api.cu", "still_step.cu", "still_tc.cu", "still_la_tc.cu", "still_static.cu"]
-HEADERS = ["still_common.cuh", "still_simt.cuh", "still_tc.h", "still_tc_ptx.cuh", os.path.join("..", "..", "include", "still.h")]
+HEADERS = ["still_common.cuh", "still_simt.cuh", "still_tc.h", "still_tc_ptx.cuh", "still_step_mma.cuh", os.path.join("..", "..", "include", "still.h")]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC", "-shared", "--threads", "0",

@@ -13,6 +13,7 @@
 //   step_merge        : combines the partials, reads out the linear branch and
 //                       applies y = (N_SA + N_LA) / (D_SA + D_LA).
 #include "still_common.cuh"
+#include "still_step_mma.cuh"
 #include "still_tc.h"
 
 #include <algorithm>
@@ -353,22 +354,52 @@ static int step_typed(const still_params_t *p, char *state, const still_state_la
 
     const long long n_routed = (lam > 0 && c_cur >= 2) ? c_cur - 1 : 0;  // chunks 0..c_cur-2
     int n_splits = 1;
-    if (n_routed > 0) {
-        long long want = (2048 + (long long)p->B * p->Hkv - 1) / ((long long)p->B * p->Hkv);
-        n_splits = (int)std::max<long long>(1, std::min<long long>({want, (long long)kMaxSplits, n_routed}));
+    if constexpr (sizeof(T) == 2) {
+        // bf16: tensor-core split-KV pass, the query heads of a KV group share every K / V row read
+        if (p->H / p->Hkv > 16) return STILL_ERR_UNSUPPORTED;  // the group's heads are the 16 rows of one MMA tile
+        const long long nb = (t + 32) / 32;  // 32-position key blocks
+        const long long groups = (long long)p->B * p->Hkv;
+        const long long want = (6 * 148 + groups - 1) / groups;  // about six waves of CTAs
+        n_splits = (int)std::max<long long>(1, std::min<long long>({want, (long long)kMaxSplits + 1, (nb + 3) / 4}));
+        dim3 grid(n_splits, p->Hkv, p->B);
+        const float scale_log2 = p->sm_scale * 1.4426950408889634f;
+        // a topk of 0 keeps nothing of the routed chunks: the kernel then sees only the local region
+        profile_mark_begin(st);
+        if (d == 64) {
+            STILL_CUDA(cudaFuncSetAttribute(step_attend_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            AttendPlan<64>::kTotal));
+            step_attend_mma_kernel<64><<<grid, 128, AttendPlan<64>::kTotal, st>>>(
+                (const __nv_bfloat16 *)kc, (const __nv_bfloat16 *)vc, sel, (const __nv_bfloat16 *)q, part, p->H, p->Hkv,
+                cap, C, lam, t, n_splits, kMaxSplits + 1, scale_log2);
+        } else {
+            STILL_CUDA(cudaFuncSetAttribute(step_attend_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            AttendPlan<128>::kTotal));
+            step_attend_mma_kernel<128><<<grid, 128, AttendPlan<128>::kTotal, st>>>(
+                (const __nv_bfloat16 *)kc, (const __nv_bfloat16 *)vc, sel, (const __nv_bfloat16 *)q, part, p->H, p->Hkv,
+                cap, C, lam, t, n_splits, kMaxSplits + 1, scale_log2);
+        }
+        profile_mark_end(st);
+        ++*launches;
+        STILL_CUDA(cudaGetLastError());
+        n_splits -= 1;  // the merge kernel reads partials 0 .. n_splits inclusive
+    } else {
+        if (n_routed > 0) {
+            long long want = (2048 + (long long)p->B * p->Hkv - 1) / ((long long)p->B * p->Hkv);
+            n_splits = (int)std::max<long long>(1, std::min<long long>({want, (long long)kMaxSplits, n_routed}));
+        }
+        const long long cps = n_routed > 0 ? (n_routed + n_splits - 1) / n_splits : 1;
+        dim3 grid(n_splits + 1, p->Hkv, p->B);
+        profile_mark_begin(st);
+        if (d == 64)
+            step_attend_kernel<T, 2><<<grid, 128, 0, st>>>(kc, vc, sel, q, part, p->H, p->Hkv, cap, C, lam, t,
+                                                           n_splits, cps, n_routed, p->sm_scale);
+        else
+            step_attend_kernel<T, 4><<<grid, 128, 0, st>>>(kc, vc, sel, q, part, p->H, p->Hkv, cap, C, lam, t,
+                                                           n_splits, cps, n_routed, p->sm_scale);
+        profile_mark_end(st);
+        ++*launches;
+        STILL_CUDA(cudaGetLastError());
     }
-    const long long cps = n_routed > 0 ? (n_routed + n_splits - 1) / n_splits : 1;
-    dim3 grid(n_splits + 1, p->Hkv, p->B);
-    profile_mark_begin(st);
-    if (d == 64)
-        step_attend_kernel<T, 2><<<grid, 128, 0, st>>>(kc, vc, sel, q, part, p->H, p->Hkv, cap, C, lam, t,
-                                                       n_splits, cps, n_routed, p->sm_scale);
-    else
-        step_attend_kernel<T, 4><<<grid, 128, 0, st>>>(kc, vc, sel, q, part, p->H, p->Hkv, cap, C, lam, t,
-                                                       n_splits, cps, n_routed, p->sm_scale);
-    profile_mark_end(st);
-    ++*launches;
-    STILL_CUDA(cudaGetLastError());
 
     step_merge_kernel<T><<<dim3(p->H, p->B), 128, 0, st>>>(part, S, z, q, g, Wq, bq, y, hdr, p->H, d, df,
                                                            n_splits, la ? 1 : 0, t);
