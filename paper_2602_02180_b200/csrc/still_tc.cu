@@ -231,6 +231,10 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             constexpr uint32_t idesc_pv = make_idesc(kBlockM, D, true);
             bool ok = mbar_wait(q_full, 0, abort_flag, status, 4);
             tc_fence_after();
+            // descriptors as low words: a k-step adds a constant (keeps this thread's instruction count low)
+            const uint32_t q_lo0 = desc_lo(smem_u32(smem + P::kQ), 0);
+            const uint32_t k_lo0 = desc_lo(smem_u32(smem + P::kK), 0);
+            const uint32_t v_lo0 = desc_lo(smem_u32(smem + P::kV), kBlockN * 128);
             int pending[2] = {-1, -1};   // stream tile whose P V product is still to be issued
             int n_done[2] = {0, 0};      // tiles processed per query tile (phase of p_full)
             auto issue_pv = [&](int x, int ip) -> bool {
@@ -238,18 +242,16 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 if (!mbar_wait(p_half + 2 * x, n_done[x] & 1, abort_flag, status, 5)) return false;
                 if (!mbar_wait(v_full + vs, (ip / P::kVStages) & 1, abort_flag, status, 6)) return false;
                 tc_fence_after();
-                const uint32_t v_addr = smem_u32(smem + P::kV + vs * P::kTileBytes);
+                const uint32_t v_lo = v_lo0 + vs * (P::kTileBytes >> 4);
+                const uint32_t d_o = tmem_base + col_o(x), a_p = tmem_base + col_s(x);
 #pragma unroll
                 for (int k = 0; k < kBlockN / 32; ++k)
-                    mma_ts(tmem_base + col_o(x), tmem_base + col_s(x) + k * 8,
-                           smem_desc(v_addr + k * 16 * 128, kBlockN * 128), idesc_pv, (n_done[x] > 0 || k > 0) ? 1u : 0u);
+                    mma_ts_lo<idesc_pv>(d_o, a_p + k * 8, v_lo + k * (16 * 128 >> 4), (n_done[x] > 0 || k > 0) ? 1u : 0u);
                 if (!mbar_wait(p_half + 2 * x + 1, n_done[x] & 1, abort_flag, status, 5)) return false;
                 tc_fence_after();
 #pragma unroll
                 for (int k = kBlockN / 32; k < kBlockN / 16; ++k)
-                    mma_ts(tmem_base + col_o(x), tmem_base + col_s(x) + k * 8,
-                           smem_desc(v_addr + k * 16 * 128, kBlockN * 128), idesc_pv, 1u);
-                tc_commit(v_empty + vs);
+                    mma_ts_lo<idesc_pv>(d_o, a_p + k * 8, v_lo + k * (16 * 128 >> 4), 1u);
                 ++n_done[x];
                 return true;
             };
@@ -258,7 +260,7 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 ok = mbar_wait(k_full + ks, (i / P::kKStages) & 1, abort_flag, status, 7);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t k_addr = smem_u32(smem + P::kK + ks * P::kTileBytes);
+                const uint32_t k_lo = k_lo0 + ks * (P::kTileBytes >> 4);
                 for (int x = 0; x < 2 && ok; ++x) {
                     const bool present = (x == 0) || st.has_b;
                     if (present && st.used_by(x, i)) {
@@ -266,21 +268,21 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                             const int ip = pending[x];
                             ok = issue_pv(x, ip);
                             if (!ok) break;
-                            // a V stage is released by two commits: pay the other tile's share if it skipped ip
-                            if (!(((1 - x) == 0 || st.has_b) && st.used_by(1 - x, ip))) tc_commit(v_empty + ip % P::kVStages);
+                            // a V stage is released by two arrivals: pay the other tile's share if it skipped ip
+                            if (!(((1 - x) == 0 || st.has_b) && st.used_by(1 - x, ip))) mbar_arrive(v_empty + ip % P::kVStages);
                         }
-                        const uint32_t q_addr = smem_u32(smem + P::kQ + x * P::kTileBytes);
+                        const uint32_t q_lo = q_lo0 + x * (P::kTileBytes >> 4), d_s = tmem_base + col_s(x);
+                        mma_ss_lo<idesc_qk, 0>(d_s, q_lo, k_lo);
 #pragma unroll
-                        for (int k = 0; k < D / 16; ++k) {
-                            const uint32_t off = (k / 4) * (kBlockM * 128) + (k % 4) * 32;
-                            mma_ss(tmem_base + col_s(x), smem_desc(q_addr + off, 0), smem_desc(k_addr + off, 0),
-                                   idesc_qk, k > 0 ? 1u : 0u);
+                        for (int k = 1; k < D / 16; ++k) {
+                            // k-step of 16 elements: 32 bytes within a 64-element swizzle atom, atoms 128 rows apart
+                            const uint32_t off = ((k / 4) * (kBlockM * 128) + (k % 4) * 32) >> 4;
+                            mma_ss_lo<idesc_qk, 1>(d_s, q_lo + off, k_lo + off);
                         }
                         tc_commit(s_full + x);
-                        tc_commit(k_empty + ks);
                         pending[x] = i;
                     } else {
-                        tc_commit(k_empty + ks);  // the share of a tile that skips this stream tile
+                        mbar_arrive(k_empty + ks);  // the share of a tile that skips this stream tile
                     }
                 }
             }
@@ -289,7 +291,6 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     const int ip = pending[x];
                     ok = issue_pv(x, ip);
                     if (!ok) break;
-                    if (!(((1 - x) == 0 || st.has_b) && st.used_by(1 - x, ip))) tc_commit(v_empty + ip % P::kVStages);
                     tc_commit(o_final + x);
                 }
             }
@@ -313,7 +314,7 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             const int lim_sel = c >= 2 ? (c - 1) * lam : 0;
             const int loc_lo = c >= 1 ? (c - 1) * C : 0;
             float m_used = -INFINITY, l_sum = 0.f;     // log2 domain
-            int n_seen = 0;
+            int n_seen = 0, prev_i = -1;
             bool ok = true;
             for (int i = 0; i < st.n_tiles && ok; ++i) {
                 if (!st.used_by(x, i)) continue;
@@ -333,6 +334,14 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 ok = mbar_wait(s_full + x, n_seen & 1, abort_flag, status, 8);
                 if (!ok) break;
                 tc_fence_after();
+                if (row_in_tile == 0) {
+                    // S_x of tile i is complete, and so is everything the MMA warp issued before it (each
+                    // tcgen05.commit costs the tensor pipe a bubble, so the ring stages are released here
+                    // instead): tile x is done with this K stage and with the V stage of its previous tile.
+                    mbar_arrive(k_empty + i % P::kKStages);
+                    if (prev_i >= 0) mbar_arrive(v_empty + prev_i % P::kVStages);
+                }
+                prev_i = i;
                 uint32_t sr[128];
                 tmem_ld32(lane_addr + col_s(x) + 0, sr + 0);
                 tmem_ld32(lane_addr + col_s(x) + 32, sr + 32);
