@@ -83,8 +83,10 @@ static FwdPlan plan_fwd(const still_params_t *p, long long N) {
     }
     if (w.tc) {
         w.sel_rows = tc_sel_rows(p, N);
-        w.ksel = take(BH * (size_t)w.sel_rows * p->d * es);
-        w.vsel = take(BH * (size_t)w.sel_rows * p->d * es);
+        if (p->topk < p->chunk) {  // with topk = chunk the salient prefix is K / V itself: no compacted copy
+            w.ksel = take(BH * (size_t)w.sel_rows * p->d * es);
+            w.vsel = take(BH * (size_t)w.sel_rows * p->d * es);
+        }
     }
     w.total = off;
     return w;

@@ -96,7 +96,7 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                    const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_ksel,
                    const __grid_constant__ CUtensorMap tm_vsel, const float *__restrict__ N_LA,
                    const float *__restrict__ D_LA, __nv_bfloat16 *__restrict__ Y, int *status, int H, int Hkv,
-                   int N, int C, int lam, int sel_rows, float scale_log2, int n_qblocks) {
+                   int N, int C, int lam, int sel_rows, int sel_identity, float scale_log2, int n_qblocks) {
     using P = SmemPlan<D>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -167,6 +167,9 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 for (int half = 0; half < D / 64; ++half)
                     tma_load_2d(smem + P::kQ + x * P::kTileBytes + half * (kBlockM * 128), &tm_q, q_full, half * 64,
                                 q_row + x * kBlockM);
+            // With topk = chunk every token is selected and the compacted arrays would be copies of K / V:
+            // the salient prefix is then read from K / V themselves (tm_ksel / tm_vsel alias tm_k / tm_v).
+            const int sel_base = sel_identity ? (b * Hkv + kvh) * N : bh * sel_rows;
             // K and V rings advance independently, each as far ahead as its free stages allow.
             bool ok = true;
             int armed_k = 0, armed_v = 0, spins = 0;
@@ -177,7 +180,7 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     const int i = armed_k, ks = i % P::kKStages;
                     if (mbar_try_wait(k_empty + ks, ((i / P::kKStages) & 1) ^ 1)) {
                         const bool sel = st.is_sel(i);
-                        const int row = sel ? bh * sel_rows + i * kBlockN : (b * Hkv + kvh) * N + st.loc_m(i) * kBlockN;
+                        const int row = sel ? sel_base + i * kBlockN : (b * Hkv + kvh) * N + st.loc_m(i) * kBlockN;
                         mbar_expect_tx(k_full + ks, P::kTileBytes);
                         for (int half = 0; half < D / 64; ++half)
                             tma_load_2d(smem + P::kK + ks * P::kTileBytes + half * (kBlockN * 128), sel ? &tm_ksel : &tm_k,
@@ -190,7 +193,7 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     const int i = armed_v, vs = i % P::kVStages;
                     if (mbar_try_wait(v_empty + vs, ((i / P::kVStages) & 1) ^ 1)) {
                         const bool sel = st.is_sel(i);
-                        const int row = sel ? bh * sel_rows + i * kBlockN : (b * Hkv + kvh) * N + st.loc_m(i) * kBlockN;
+                        const int row = sel ? sel_base + i * kBlockN : (b * Hkv + kvh) * N + st.loc_m(i) * kBlockN;
                         mbar_expect_tx(v_full + vs, P::kTileBytes);
                         for (int half = 0; half < D / 64; ++half)
                             tma_load_2d(smem + P::kV + vs * P::kTileBytes + half * (kBlockN * 128), sel ? &tm_vsel : &tm_v,
@@ -239,8 +242,9 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             int n_done[2] = {0, 0};      // tiles processed per query tile (phase of p_full)
             auto issue_pv = [&](int x, int ip) -> bool {
                 const int vs = ip % P::kVStages;
-                if (!mbar_wait(p_half + 2 * x, n_done[x] & 1, abort_flag, status, 5)) return false;
+                // (V has normally arrived long ago: checking it first hides the check behind the wait for P)
                 if (!mbar_wait(v_full + vs, (ip / P::kVStages) & 1, abort_flag, status, 6)) return false;
+                if (!mbar_wait(p_half + 2 * x, n_done[x] & 1, abort_flag, status, 5)) return false;
                 tc_fence_after();
                 const uint32_t v_lo = v_lo0 + vs * (P::kTileBytes >> 4);
                 const uint32_t d_o = tmem_base + col_o(x), a_p = tmem_base + col_s(x);
@@ -673,7 +677,8 @@ int launch_tc(const still_params_t *p, long long N, const void *Q, const void *K
     using bf = __nv_bfloat16;
     const long long T = (N + p->chunk - 1) / p->chunk, BH = (long long)p->B * p->H;
     const long long n_idx = T * p->topk;
-    {
+    const bool identity = p->topk == p->chunk;  // the selection of every chunk is the chunk itself
+    if (!identity) {
         dim3 grid((unsigned)((sel_rows + 7) / 8), (unsigned)BH);
         compact_kernel<D><<<grid, 256, 0, st>>>((const bf *)K, (const bf *)V, sel_idx, (bf *)k_sel, (bf *)v_sel, p->H,
                                                p->Hkv, N, n_idx, sel_rows);
@@ -684,8 +689,8 @@ int launch_tc(const still_params_t *p, long long N, const void *Q, const void *K
     if (!make_map(&tq, Q, (unsigned long long)BH * N, D) ||
         !make_map(&tk, K, (unsigned long long)p->B * p->Hkv * N, D) ||
         !make_map(&tv, V, (unsigned long long)p->B * p->Hkv * N, D) ||
-        !make_map(&tks, k_sel, (unsigned long long)BH * sel_rows, D) ||
-        !make_map(&tvs, v_sel, (unsigned long long)BH * sel_rows, D))
+        !make_map(&tks, identity ? K : k_sel, identity ? (unsigned long long)p->B * p->Hkv * N : (unsigned long long)BH * sel_rows, D) ||
+        !make_map(&tvs, identity ? V : v_sel, identity ? (unsigned long long)p->B * p->Hkv * N : (unsigned long long)BH * sel_rows, D))
         return STILL_ERR_CUDA;
     const int n_qblocks = (int)((N + 2 * kBlockM - 1) / (2 * kBlockM));
     if (cudaFuncSetAttribute(sa_merge_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -694,7 +699,7 @@ int launch_tc(const still_params_t *p, long long N, const void *Q, const void *K
     dim3 grid((unsigned)n_qblocks, (unsigned)BH);
     profile_mark_begin(st);
     sa_merge_tc_kernel<D><<<grid, kThreads, SmemPlan<D>::kAlloc, st>>>(
-        tq, tk, tv, tks, tvs, N_LA, D_LA, (bf *)Y, status, p->H, p->Hkv, (int)N, p->chunk, p->topk, (int)sel_rows,
+        tq, tk, tv, tks, tvs, N_LA, D_LA, (bf *)Y, status, p->H, p->Hkv, (int)N, p->chunk, p->topk, (int)sel_rows, identity ? 1 : 0,
         p->sm_scale * 1.4426950408889634f, n_qblocks);
     profile_mark_end(st);
     ++*launches;
