@@ -159,7 +159,7 @@ def run_reference(args, w, lam, rank, world):
 
     cores = multiprocessing.cpu_count()
     n_heads = max(1, min(cores, w.B * w.H))
-    n_rows = 48 if w.N > 8192 else 256
+    n_rows = 160 if w.N > 8192 else 256
     times = []
     for i in range(args.warmup + args.steps):
         total, threads, sample, spent = oracle_sample(w, lam, n_heads, n_rows)
@@ -330,7 +330,7 @@ def bench_prefill(args, w, lam, still, synth, torch, dist, dev, rank, world):
         import multiprocessing
 
         n_heads = max(1, min(multiprocessing.cpu_count(), w.B * w.H))
-        total, threads, sample, _ = oracle_sample(w, lam, n_heads, 48 if w.N > 8192 else 256)
+        total, threads, sample, _ = oracle_sample(w, lam, n_heads, 160 if w.N > 8192 else 256)
         cpu = {"value": w.B * w.N / total, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample}
 
     return {

@@ -84,6 +84,8 @@ def _decode_case(w, n0, n_steps, gate=False):
         (1, 8, 2, 128, 64, 64, 130, 66),   # lambda = C
         (1, 2, 1, 64, 32, 8, 0, 100),      # decode from an empty state
         (1, 2, 2, 128, 128, 32, 300, 90),
+        (1, 16, 1, 64, 32, 8, 90, 50),     # sixteen query heads on one KV head
+        (1, 12, 2, 128, 64, 16, 200, 70),  # six heads per group
     ],
 )
 def test_decode_matches_oracle(dtype, B, H, Hkv, d, C, k, n0, steps):

@@ -49,6 +49,21 @@ def test_small_shapes(dtype, B, H, Hkv, d, N, C, k):
                     G=r["G"], bq=r["bq"], bk=r["bk"])
 
 
+def test_feature_width_smaller_than_head_dim():
+    # d_f = 64 with d = 128: feature dim d' = 128 (other template instance of the NP-Map and scan kernels)
+    w = _small("t", "bf16", 1, 4, 2, 128, 64 * 7 + 5, 64, 16)
+    Q, K, V = synth.make_qkv(w, "cuda")
+    g = torch.Generator(device="cuda").manual_seed(11)
+    Wq = (torch.randn(w.H, w.d, 64, generator=g, device="cuda") * 0.02).to(torch.bfloat16)
+    Wk = (torch.randn(w.Hkv, w.d, 64, generator=g, device="cuda") * 0.02).to(torch.bfloat16)
+    p = still.StillParams(w.B, w.H, w.Hkv, w.d, w.C, w.k, torch.bfloat16, d_f=64)
+    Y, scores, sel = still.hybrid_attn_fwd(p, Q, K, V, Wq, Wk)
+    torch.cuda.synchronize()
+    heads = U.sample_heads(w, 4)
+    U.check_selection(scores, sel, w.C, w.k, heads)
+    U.check_outputs(w, Q, K, V, Wq, Wk, Y, scores, sel, heads)
+
+
 def test_paper_literal_scale_one():
     # sm_scale = 1 is the main text's exp(q k^T); inputs are scaled down so the softmaxes stay soft.
     w = _small("t", "fp32", 1, 2, 2, 64, 256, 64, 16)
