@@ -137,7 +137,7 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         for (int i = 0; i < P::kKStages; ++i) { mbar_init(k_full + i, 1); mbar_init(k_empty + i, 2); }
         for (int i = 0; i < P::kVStages; ++i) { mbar_init(v_full + i, 1); mbar_init(v_empty + i, 2); }
         for (int i = 0; i < 2; ++i) { mbar_init(s_full + i, 1); mbar_init(o_final + i, 1); }
-        for (int i = 0; i < 4; ++i) mbar_init(p_half + i, 128);
+        for (int i = 0; i < 4; ++i) mbar_init(p_half + i, 4);  // one arrival per softmax warp
         mbar_init(drain, 1);
         *abort_flag = 0;
         fence_barrier_init();
@@ -408,7 +408,8 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                             // the first half of P has had time to land: hand it to the MMA warp
                             tmem_wait_st();
                             tc_fence_before();
-                            mbar_arrive(p_half + 2 * x);
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(p_half + 2 * x);
                         }
                     }
                     tmem_st32(lane_addr + col_s(x) + q * 32, pk);
@@ -416,7 +417,8 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 l_sum += acc.x + acc.y;
                 tmem_wait_st();
                 tc_fence_before();
-                mbar_arrive(p_half + 2 * x + 1);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(p_half + 2 * x + 1);
                 ++n_seen;
             }
             // ---- epilogue: y = (O e^{m-ms} + e^{-ms} N_LA) / (l e^{m-ms} + e^{-ms} D_LA), ms = max(m, 0)
