@@ -93,6 +93,13 @@ def test_decode_matches_oracle(dtype, B, H, Hkv, d, C, k, n0, steps):
     _decode_case(w, n0, steps, gate=(k not in (0, C)))
 
 
+def test_c5_full_size_sampled():
+    # The decode workload as benchmarked: batch 64, 32768-token prefix summarised by the prefill into the
+    # decode state, then a few steps; sampled (batch, head) pairs against the oracle.
+    w = synth.WORKLOADS["c5"]
+    _decode_case(w, w.N, 3)
+
+
 def test_state_full_and_mismatch():
     w = synth.Workload("t", 1, 2, 2, 64, 64, 32, 8, "bf16", "iid", 5)
     p = U.params_of(w)
