@@ -57,7 +57,7 @@ __device__ __forceinline__ void mma_ts_tf32(uint32_t d_tmem, uint32_t a_tmem, ui
 // NP-Map
 // ------------------------------------------------------------------------------------------
 template <int D, int DF, typename TOut>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(192, 3)
 npmap_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
                 const __nv_bfloat16 *__restrict__ bias, TOut *__restrict__ phi, int *status, int heads, int N) {
     constexpr int kXBytes = 128 * D * 2, kWBytes = D * DF * 2;
@@ -131,54 +131,81 @@ npmap_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
         ok = __all_sync(0xffffffffu, ok);
         if (ok) {
             tc_fence_after();
-            float f[DF];
+            // Three passes over the row of f in tensor memory, 32 columns at a time, so that the row is
+            // never held in registers (several CTAs per SM then overlap their load / MMA / epilogue
+            // phases): norms and extrema, the two softmax denominators, the features themselves.
+            const __nv_bfloat16 *bh_ = bias != nullptr ? bias + (long long)hd * DF : nullptr;
+            float nf2 = 0.f, fmax_ = -INFINITY, fmin_ = INFINITY;
+#pragma unroll 1
+            for (int q = 0; q < DF / 32; ++q) {
+                uint32_t v[32];
+                tmem_ld32(taddr + q * 32, v);
+                tmem_wait_ld();
 #pragma unroll
-            for (int q = 0; q < DF / 32; ++q) tmem_ld32(taddr + q * 32, reinterpret_cast<uint32_t *>(f) + q * 32);
-            tmem_wait_ld();
-            float nf2 = 0.f;
-#pragma unroll
-            for (int j = 0; j < DF; ++j) {
-                if (bias != nullptr) f[j] += __bfloat162float(bias[(long long)hd * DF + j]);
-                nf2 = fmaf(f[j], f[j], nf2);
+                for (int j = 0; j < 32; ++j) {
+                    float x = __uint_as_float(v[j]);
+                    if (bh_ != nullptr) x += __bfloat162float(bh_[q * 32 + j]);
+                    nf2 = fmaf(x, x, nf2);
+                    fmax_ = fmaxf(fmax_, x);
+                    fmin_ = fminf(fmin_, x);
+                }
             }
-            const float ratio = sqrtf(nx2) / fmaxf(sqrtf(nf2), 1e-12f) * 1.4426950408889634f;  // u in the log2 domain
-            float umax = -INFINITY, umin = INFINITY;
-#pragma unroll
-            for (int j = 0; j < DF; ++j) {
-                f[j] *= ratio;
-                umax = fmaxf(umax, f[j]);
-                umin = fminf(umin, f[j]);
-            }
+            // u = f * ratio in the log2 domain; ratio > 0, so the extrema of u are those of f
+            const float ratio = sqrtf(nx2) / fmaxf(sqrtf(nf2), 1e-12f) * 1.4426950408889634f;
+            const float umax = fmax_ * ratio, umin = fmin_ * ratio;
             float zp = 0.f, zn = 0.f;
+#pragma unroll 1
+            for (int q = 0; q < DF / 32; ++q) {
+                uint32_t v[32];
+                tmem_ld32(taddr + q * 32, v);
+                tmem_wait_ld();
 #pragma unroll
-            for (int j = 0; j < DF; ++j) {
-                zp += ex2(f[j] - umax);
-                zn += ex2(umin - f[j]);
+                for (int j = 0; j < 32; ++j) {
+                    float x = __uint_as_float(v[j]);
+                    if (bh_ != nullptr) x += __bfloat162float(bh_[q * 32 + j]);
+                    const float u = x * ratio;
+                    zp += ex2(u - umax);
+                    zn += ex2(umin - u);
+                }
             }
             const float ip = 1.f / zp, in = 1.f / zn;
-            if (R0 + r < N) {
-                TOut *out = phi + (row0 + r) * (2 * DF);
-                if constexpr (sizeof(TOut) == 4) {
+            const bool live = R0 + r < N;
+            TOut *out = phi + (row0 + r) * (2 * DF);
+#pragma unroll 1
+            for (int q = 0; q < DF / 32; ++q) {
+                uint32_t v[32];
+                tmem_ld32(taddr + q * 32, v);
+                tmem_wait_ld();
+                float u[32];
 #pragma unroll
-                    for (int j = 0; j < DF; j += 4) {
-                        *reinterpret_cast<float4 *>(out + j) =
-                            make_float4(ex2(f[j] - umax) * ip, ex2(f[j + 1] - umax) * ip, ex2(f[j + 2] - umax) * ip,
-                                        ex2(f[j + 3] - umax) * ip);
-                        *reinterpret_cast<float4 *>(out + DF + j) =
-                            make_float4(ex2(umin - f[j]) * in, ex2(umin - f[j + 1]) * in, ex2(umin - f[j + 2]) * in,
-                                        ex2(umin - f[j + 3]) * in);
-                    }
-                } else {
+                for (int j = 0; j < 32; ++j) {
+                    float x = __uint_as_float(v[j]);
+                    if (bh_ != nullptr) x += __bfloat162float(bh_[q * 32 + j]);
+                    u[j] = x * ratio;
+                }
+                if (live) {
+                    if constexpr (sizeof(TOut) == 4) {
 #pragma unroll
-                    for (int j = 0; j < DF; j += 8) {
-                        uint32_t pp[4], nn[4];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            pp[e] = pack_bf16(ex2(f[j + 2 * e] - umax) * ip, ex2(f[j + 2 * e + 1] - umax) * ip);
-                            nn[e] = pack_bf16(ex2(umin - f[j + 2 * e]) * in, ex2(umin - f[j + 2 * e + 1]) * in);
+                        for (int j = 0; j < 32; j += 4) {
+                            *reinterpret_cast<float4 *>(out + q * 32 + j) =
+                                make_float4(ex2(u[j] - umax) * ip, ex2(u[j + 1] - umax) * ip, ex2(u[j + 2] - umax) * ip,
+                                            ex2(u[j + 3] - umax) * ip);
+                            *reinterpret_cast<float4 *>(out + DF + q * 32 + j) =
+                                make_float4(ex2(umin - u[j]) * in, ex2(umin - u[j + 1]) * in, ex2(umin - u[j + 2]) * in,
+                                            ex2(umin - u[j + 3]) * in);
                         }
-                        *reinterpret_cast<uint4 *>(out + j) = make_uint4(pp[0], pp[1], pp[2], pp[3]);
-                        *reinterpret_cast<uint4 *>(out + DF + j) = make_uint4(nn[0], nn[1], nn[2], nn[3]);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 8) {
+                            uint32_t pp[4], nn[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                pp[e] = pack_bf16(ex2(u[j + 2 * e] - umax) * ip, ex2(u[j + 2 * e + 1] - umax) * ip);
+                                nn[e] = pack_bf16(ex2(umin - u[j + 2 * e]) * in, ex2(umin - u[j + 2 * e + 1]) * in);
+                            }
+                            *reinterpret_cast<uint4 *>(out + q * 32 + j) = make_uint4(pp[0], pp[1], pp[2], pp[3]);
+                            *reinterpret_cast<uint4 *>(out + DF + q * 32 + j) = make_uint4(nn[0], nn[1], nn[2], nn[3]);
+                        }
                     }
                 }
             }
