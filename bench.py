@@ -387,8 +387,12 @@ def bench_decode(args, w, lam, still, synth, torch, dist, dev, rank, world):
     ms_step = ms_total / n_steps
     peaks = measured_peaks()
     es = 2
-    n_hist = (t // w.C - 1) * lam if lam > 0 else 0
-    # K and V rows of the salient history once per KV head, the local region, and the LA state
+    # K and V rows of the routed history that at least one query head of the KV group selected (expected
+    # size of the union of the group's selections: 1 - (1 - lam/C)^group of the rows; all rows when
+    # lam = C), read once per KV head, plus the local region and, when it is in use, the LA state
+    rep = w.H // w.Hkv
+    union = 1.0 - (1.0 - lam / w.C) ** rep if lam > 0 else 0.0
+    n_hist = (t // w.C - 1) * w.C * union
     by = w.B * w.Hkv * (n_hist + 2 * w.C) * w.d * es * 2 + (w.B * w.H * 2 * w.d_f * (w.d + 1) * 4 if lam < w.C else 0)
     k_ms = statistics.mean(kernel_ms) if kernel_ms else ms_step
     ach = by / (k_ms * 1e-3) / 1e9

@@ -105,12 +105,15 @@ size_t still_state_bytes(const still_params_t *p, int64_t max_tokens);
  *   sel_idx  : [B, H, capacity / chunk, topk] int32 -- salient positions of each
  *              routed chunk, ascending, -1 padded (rows of chunks not yet routed
  *              are unspecified).
+ *   sel_mask : [B, H, capacity / chunk, chunk / 32] uint32 -- the same selection as
+ *              bit masks: bit j of word w of chunk c is set when position
+ *              c * chunk + 32 w + j is selected (what the decode kernel reads).
  *   S        : [B, H, 2 d_f, d] fp32 -- KV state s_t.
  *   z        : [B, H, 2 d_f] fp32 -- normaliser z_t.
  *   scratch  : split-KV partial results of the step kernel.
  */
 typedef struct still_state_layout {
-    size_t header, k_cache, v_cache, score, sel_idx, S, z, scratch, total;
+    size_t header, k_cache, v_cache, score, sel_idx, sel_mask, S, z, scratch, total;
     int64_t capacity; /* max_tokens rounded up to a multiple of chunk */
 } still_state_layout_t;
 int still_state_layout(const still_params_t *p, int64_t max_tokens, still_state_layout_t *out);

@@ -29,7 +29,7 @@ class _CParams(ctypes.Structure):
 
 class _CStateLayout(ctypes.Structure):
     _fields_ = [(n, ctypes.c_size_t) for n in
-                ("header", "k_cache", "v_cache", "score", "sel_idx", "S", "z", "scratch", "total")] + [
+                ("header", "k_cache", "v_cache", "score", "sel_idx", "sel_mask", "S", "z", "scratch", "total")] + [
         ("capacity", ctypes.c_int64)]
 
 

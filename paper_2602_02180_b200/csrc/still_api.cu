@@ -109,6 +109,7 @@ static int plan_state(const still_params_t *p, long long max_tokens, still_state
     L->v_cache = take(BHkv * (size_t)cap * p->d * es);
     L->score = take(BH * (size_t)cap * 4);
     L->sel_idx = take(BH * (size_t)(cap / p->chunk) * (size_t)std::max(p->topk, 1) * 4);
+    L->sel_mask = take(BH * (size_t)(cap / p->chunk) * (size_t)(p->chunk / 32) * 4);
     L->S = take(BH * dp * p->d * 4);
     L->z = take(BH * dp * 4);
     L->scratch = take(step_scratch_bytes(p, cap));
@@ -136,6 +137,27 @@ __global__ void write_header_kernel(int32_t *hdr, still_params_t p, long long ca
         hdr[10] = (int32_t)(cap & 0xffffffffll); hdr[11] = (int32_t)(cap >> 32);
         hdr[12] = (int32_t)(t & 0xffffffffll); hdr[13] = (int32_t)(t >> 32);
         hdr[14] = 0; hdr[15] = 0;
+    }
+}
+
+// Selection of every chunk as bit masks for the decode state: one warp per (head, chunk); bit j of
+// word w is set when position chunk * C + 32 w + j is among the chunk's selected positions.
+__global__ void sel_mask_kernel(const int32_t *__restrict__ sel_idx, uint32_t *__restrict__ sel_mask, long long BH,
+                                long long T, long long capT, int C, int lam) {
+    const long long wid = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (wid >= BH * T) return;
+    const int lane = threadIdx.x & 31;
+    const long long bh = wid / T, c = wid % T;
+    const int32_t *si = sel_idx + (bh * T + c) * lam;
+    for (int w = 0; w < C / 32; ++w) {
+        const long long p0 = c * C + 32ll * w;
+        uint32_t bits = 0u;
+        for (int i = lane; i < lam; i += 32) {
+            const long long p = si[i];
+            if (p >= p0 && p < p0 + 32) bits |= 1u << (int)(p - p0);
+        }
+        bits = __reduce_or_sync(0xffffffffu, bits);
+        if (lane == 0) sel_mask[(bh * capT + c) * (C / 32) + w] = bits;
     }
 }
 
@@ -301,6 +323,14 @@ static int fwd_typed(const still_params_t *p, long long N, const T *Q, const T *
             STILL_CUDA(cudaMemcpy2DAsync(state + L.sel_idx, (size_t)(L.capacity / p->chunk) * p->topk * 4,
                                          sel, (size_t)w.T * p->topk * 4, (size_t)w.T * p->topk * 4, BH,
                                          cudaMemcpyDeviceToDevice, st));
+        if (p->topk > 0) {
+            const long long units = (long long)BH * w.T;
+            sel_mask_kernel<<<(unsigned)((units + 7) / 8), 256, 0, st>>>(
+                sel, reinterpret_cast<uint32_t *>(state + L.sel_mask), (long long)BH, w.T, L.capacity / p->chunk,
+                p->chunk, p->topk);
+            ++g_launches;
+            STILL_CUDA(cudaGetLastError());
+        }
         write_header_kernel<<<1, 32, 0, st>>>(reinterpret_cast<int32_t *>(state + L.header), *p,
                                               L.capacity, N);
         ++g_launches;

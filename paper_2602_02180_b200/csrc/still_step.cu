@@ -101,8 +101,8 @@ __global__ void step_append_score_kernel(T *__restrict__ kc, T *__restrict__ vc,
 template <typename T>
 __global__ void __launch_bounds__(256)
 step_route_kernel(const T *__restrict__ kc, const T *__restrict__ vc, const float *__restrict__ score,
-                  int32_t *__restrict__ sel_idx, float *__restrict__ S, float *__restrict__ z,
-                  const T *__restrict__ Wk, const T *__restrict__ bk, int H, int Hkv, long long cap,
+                  int32_t *__restrict__ sel_idx, uint32_t *__restrict__ sel_mask, float *__restrict__ S,
+                  float *__restrict__ z, const T *__restrict__ Wk, const T *__restrict__ bk, int H, int Hkv, long long cap,
                   int d, int df, int C, int lam, long long cr) {
     extern __shared__ float smem[];
     const int dp = 2 * df;
@@ -121,6 +121,11 @@ step_route_kernel(const T *__restrict__ kc, const T *__restrict__ vc, const floa
     __syncthreads();
     if (lam > 0) select_chunk(sc, flag, C, C, lam, base, sel_idx + (bh * (cap / C) + cr) * lam);
     __syncthreads();
+    if (threadIdx.x < C / 32) {  // the same selection as bit masks (read by the split-KV pass)
+        uint32_t bits = 0u;
+        for (int j = 0; j < 32; ++j) bits |= (flag[threadIdx.x * 32 + j] ? 1u : 0u) << j;
+        sel_mask[(bh * (cap / C) + cr) * (C / 32) + threadIdx.x] = bits;
+    }
     if (lam >= C) return;  // nothing goes to the linear branch
     const T *kh = kc + (((long long)b * Hkv + kv) * cap + base) * d;
     const T *vh = vc + (((long long)b * Hkv + kv) * cap + base) * d;
@@ -331,6 +336,7 @@ static int step_typed(const still_params_t *p, char *state, const still_state_la
     T *kc = reinterpret_cast<T *>(state + L->k_cache), *vc = reinterpret_cast<T *>(state + L->v_cache);
     float *score = reinterpret_cast<float *>(state + L->score);
     int32_t *sel = reinterpret_cast<int32_t *>(state + L->sel_idx);
+    uint32_t *smask = reinterpret_cast<uint32_t *>(state + L->sel_mask);
     float *S = reinterpret_cast<float *>(state + L->S), *z = reinterpret_cast<float *>(state + L->z);
     float *part = reinterpret_cast<float *>(state + L->scratch);
     int32_t *hdr = reinterpret_cast<int32_t *>(state + L->header);
@@ -346,7 +352,7 @@ static int step_typed(const still_params_t *p, char *state, const still_state_la
         size_t smem = ((size_t)C * 2 * df + (size_t)C * d + 8 * (size_t)d + C) * 4 + (size_t)C * 4;
         STILL_CUDA(cudaFuncSetAttribute(step_route_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)smem));
-        step_route_kernel<T><<<dim3(p->H, p->B), 256, smem, st>>>(kc, vc, score, sel, S, z, Wk, bk, p->H,
+        step_route_kernel<T><<<dim3(p->H, p->B), 256, smem, st>>>(kc, vc, score, sel, smask, S, z, Wk, bk, p->H,
                                                                   p->Hkv, cap, d, df, C, lam, c_cur - 2);
         ++*launches;
         STILL_CUDA(cudaGetLastError());
@@ -369,13 +375,13 @@ static int step_typed(const still_params_t *p, char *state, const still_state_la
             STILL_CUDA(cudaFuncSetAttribute(step_attend_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                             AttendPlan<64>::kTotal));
             step_attend_mma_kernel<64><<<grid, 128, AttendPlan<64>::kTotal, st>>>(
-                (const __nv_bfloat16 *)kc, (const __nv_bfloat16 *)vc, sel, (const __nv_bfloat16 *)q, part, p->H, p->Hkv,
+                (const __nv_bfloat16 *)kc, (const __nv_bfloat16 *)vc, smask, (const __nv_bfloat16 *)q, part, p->H, p->Hkv,
                 cap, C, lam, t, n_splits, kMaxSplits + 1, scale_log2);
         } else {
             STILL_CUDA(cudaFuncSetAttribute(step_attend_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                             AttendPlan<128>::kTotal));
             step_attend_mma_kernel<128><<<grid, 128, AttendPlan<128>::kTotal, st>>>(
-                (const __nv_bfloat16 *)kc, (const __nv_bfloat16 *)vc, sel, (const __nv_bfloat16 *)q, part, p->H, p->Hkv,
+                (const __nv_bfloat16 *)kc, (const __nv_bfloat16 *)vc, smask, (const __nv_bfloat16 *)q, part, p->H, p->Hkv,
                 cap, C, lam, t, n_splits, kMaxSplits + 1, scale_log2);
         }
         profile_mark_end(st);

@@ -4,7 +4,7 @@
 // range of 32-position key blocks; the query heads of the group (at most 16) are the rows of one
 // m16n8k16 tensor-core tile, so the K / V rows are read once for the whole group.  Which rows a
 // query head sees is a per-head membership mask: for a position in a routed chunk, whether the
-// head's selection (sel_idx) contains it; for the two-chunk local region, every position up to the
+// head's selection (the sel_mask words of the decode state) contains it; for the two-chunk local region, every position up to the
 // new token.  Whole key blocks are streamed (coalesced 16-byte cp.async into padded shared-memory
 // rows, two stages per warp) and rows a head did not select get weight zero; with topk = chunk
 // that is exactly the salient cache, with a smaller topk a block is still read once for the
@@ -69,7 +69,7 @@ struct AttendPlan {
 template <int D>
 __global__ void __launch_bounds__(128)
 step_attend_mma_kernel(const __nv_bfloat16 *__restrict__ kc, const __nv_bfloat16 *__restrict__ vc,
-                       const int32_t *__restrict__ sel_idx, const __nv_bfloat16 *__restrict__ q,
+                       const uint32_t *__restrict__ sel_mask, const __nv_bfloat16 *__restrict__ q,
                        float *__restrict__ part, int H, int Hkv, long long cap, int C, int lam, long long t,
                        int n_splits, int max_splits, float scale_log2) {
     using P = AttendPlan<D>;
@@ -143,18 +143,14 @@ step_attend_mma_kernel(const __nv_bfloat16 *__restrict__ kc, const __nv_bfloat16
                 vis[0] = g < rep ? 0xffffffffu : 0u;   // every token of a routed chunk was selected
                 vis[1] = g + 8 < rep ? 0xffffffffu : 0u;
             } else if (lam > 0) {
-                const int chunk = (int)(p0 / C);
-                for (int r = 0; r < rep; ++r) {
-                    const int32_t *si = sel_idx + ((((long long)b * H + (long long)kv * rep + r) * n_chunk_cap) + chunk) * lam;
-                    uint32_t bits = 0u;
-                    for (int i = lane; i < lam; i += 32) {
-                        const long long p = si[i];
-                        if (p >= p0 && p < p0 + 32) bits |= 1u << (int)(p - p0);
-                    }
-                    bits = __reduce_or_sync(0xffffffffu, bits);
-                    if (r == g) vis[0] = bits;
-                    if (r == g + 8) vis[1] = bits;
-                }
+                // selection of the block's chunk as bit masks (written when the chunk was routed): lane r
+                // fetches the word of head r, rows g and g + 8 take theirs by shuffle
+                const int chunk = (int)(p0 / C), word = (int)((p0 % C) / 32);
+                uint32_t mine = 0u;
+                if (lane < rep)
+                    mine = sel_mask[(((long long)b * H + (long long)kv * rep + lane) * n_chunk_cap + chunk) * (C / 32) + word];
+                vis[0] = __shfl_sync(0xffffffffu, mine, g);
+                vis[1] = __shfl_sync(0xffffffffu, mine, g + 8);
             }
         }
         cp_async_wait<1>();

@@ -50,7 +50,7 @@ def test_validation_and_sizes(lib):
         assert still.state_bytes(bad, 1024) == 0
     lay = still.state_layout(still.StillParams(1, 4, 2, 64, 64, 16), 1000)
     assert lay["capacity"] == 1024 and lay["total"] == still.state_bytes(still.StillParams(1, 4, 2, 64, 64, 16), 1000)
-    order = [lay[k] for k in ("header", "k_cache", "v_cache", "score", "sel_idx", "S", "z", "scratch", "total")]
+    order = [lay[k] for k in ("header", "k_cache", "v_cache", "score", "sel_idx", "sel_mask", "S", "z", "scratch", "total")]
     assert order == sorted(order) and all(o % 256 == 0 for o in order)
     with pytest.raises(still.StillError):
         still.state_layout(still.StillParams(1, 4, 3, 64, 64, 16), 1000)
