@@ -473,23 +473,103 @@ int still_hybrid_attn_fwd_host(const still_params_t *p, int64_t N, const void *h
     char *dsc = take(scb), *dsi = take(sib);
     char *ws = a + off;
     const size_t ws_bytes = arena_bytes - off;
-    STILL_CUDA(cudaMemcpyAsync(dQ, hQ, qb, cudaMemcpyHostToDevice, st));
-    STILL_CUDA(cudaMemcpyAsync(dK, hK, kvb, cudaMemcpyHostToDevice, st));
-    STILL_CUDA(cudaMemcpyAsync(dV, hV, kvb, cudaMemcpyHostToDevice, st));
-    if (hG) STILL_CUDA(cudaMemcpyAsync(dG, hG, qb, cudaMemcpyHostToDevice, st));
+    // Weights first, on the caller's stream.
     if (hWq) STILL_CUDA(cudaMemcpyAsync(dWq, hWq, wqb, cudaMemcpyHostToDevice, st));
     if (hbq) STILL_CUDA(cudaMemcpyAsync(dbq, hbq, bqb, cudaMemcpyHostToDevice, st));
     if (hWk) STILL_CUDA(cudaMemcpyAsync(dWk, hWk, wkb, cudaMemcpyHostToDevice, st));
     if (hbk) STILL_CUDA(cudaMemcpyAsync(dbk, hbk, bkb, cudaMemcpyHostToDevice, st));
-    rc = still_hybrid_attn_fwd(p, N, dQ, dK, dV, hG ? dG : nullptr, hWq ? dWq : nullptr,
-                               hbq ? dbq : nullptr, hWk ? dWk : nullptr, hbk ? dbk : nullptr, dY,
-                               reinterpret_cast<float *>(dsc), reinterpret_cast<int32_t *>(dsi),
-                               nullptr, 0, ws, ws_bytes, cuda_stream);
+
+    // The (batch, KV-head group) units are independent, so the call is cut into up to eight parts --
+    // contiguous ranges of KV heads of one batch entry with their query heads -- and pipelined: the
+    // host-to-device copies of part i+1 and the device-to-host copies of part i-1 run on two side
+    // streams while part i computes on the caller's stream (PCIe is full duplex, and the copies are as
+    // long as the compute at the benchmark shapes).
+    static thread_local cudaStream_t s_in = nullptr, s_out = nullptr;
+    if (!s_in) {
+        STILL_CUDA(cudaStreamCreateWithFlags(&s_in, cudaStreamNonBlocking));
+        STILL_CUDA(cudaStreamCreateWithFlags(&s_out, cudaStreamNonBlocking));
+    }
+    const int rep = p->H / p->Hkv;
+    int g = std::max(1, p->Hkv * p->B / 8);          // KV heads per part
+    while (p->Hkv % g != 0) --g;
+    const int parts_per_b = p->Hkv / g, n_parts = p->B * parts_per_b;
+    constexpr int kMaxParts = 64;
+    const size_t sc_part_bytes = (size_t)g * rep * N * 4, si_part_bytes = (size_t)g * rep * T * std::max(p->topk, 1) * 4;
+    if (n_parts > kMaxParts || sc_part_bytes % 16 != 0 || si_part_bytes % 16 != 0) {
+        // too many parts for the fixed event table, or a part's scores / indices would not start on a
+        // 16-byte boundary (N not a multiple of 4): plain copy - compute - copy
+        STILL_CUDA(cudaMemcpyAsync(dQ, hQ, qb, cudaMemcpyHostToDevice, st));
+        STILL_CUDA(cudaMemcpyAsync(dK, hK, kvb, cudaMemcpyHostToDevice, st));
+        STILL_CUDA(cudaMemcpyAsync(dV, hV, kvb, cudaMemcpyHostToDevice, st));
+        if (hG) STILL_CUDA(cudaMemcpyAsync(dG, hG, qb, cudaMemcpyHostToDevice, st));
+        rc = still_hybrid_attn_fwd(p, N, dQ, dK, dV, hG ? dG : nullptr, hWq ? dWq : nullptr, hbq ? dbq : nullptr,
+                                   hWk ? dWk : nullptr, hbk ? dbk : nullptr, dY, reinterpret_cast<float *>(dsc),
+                                   reinterpret_cast<int32_t *>(dsi), nullptr, 0, ws, ws_bytes, cuda_stream);
+        if (rc != STILL_OK) return rc;
+        STILL_CUDA(cudaMemcpyAsync(hY, dY, qb, cudaMemcpyDeviceToHost, st));
+        if (hscores) STILL_CUDA(cudaMemcpyAsync(hscores, dsc, scb, cudaMemcpyDeviceToHost, st));
+        if (hsel_idx && p->topk > 0) STILL_CUDA(cudaMemcpyAsync(hsel_idx, dsi, sib, cudaMemcpyDeviceToHost, st));
+        STILL_CUDA(cudaStreamSynchronize(st));
+        return STILL_OK;
+    }
+    cudaEvent_t ev_start, ev_in[kMaxParts], ev_done[kMaxParts];
+    STILL_CUDA(cudaEventCreateWithFlags(&ev_start, cudaEventDisableTiming));
+    for (int i = 0; i < n_parts; ++i) {
+        STILL_CUDA(cudaEventCreateWithFlags(&ev_in[i], cudaEventDisableTiming));
+        STILL_CUDA(cudaEventCreateWithFlags(&ev_done[i], cudaEventDisableTiming));
+    }
+    auto cleanup = [&]() {
+        cudaEventDestroy(ev_start);
+        for (int i = 0; i < n_parts; ++i) {
+            cudaEventDestroy(ev_in[i]);
+            cudaEventDestroy(ev_done[i]);
+        }
+    };
+    // the side streams start after what the caller has already enqueued (and after the weights)
+    STILL_CUDA(cudaEventRecord(ev_start, st));
+    STILL_CUDA(cudaStreamWaitEvent(s_in, ev_start, 0));
+    still_params_t sub = *p;
+    sub.B = 1;
+    sub.Hkv = g;
+    sub.H = g * rep;
+    const size_t q_part = (size_t)g * rep * N * p->d * es, kv_part = (size_t)g * N * p->d * es;
+    const size_t sc_part = (size_t)g * rep * N * 4, si_part = (size_t)g * rep * T * std::max(p->topk, 1) * 4;
+    const char *cQ = static_cast<const char *>(hQ), *cK = static_cast<const char *>(hK), *cV = static_cast<const char *>(hV);
+    const char *cG = static_cast<const char *>(hG);
+    for (int i = 0; i < n_parts; ++i) {
+        cudaError_t e = cudaMemcpyAsync(dQ + i * q_part, cQ + i * q_part, q_part, cudaMemcpyHostToDevice, s_in);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(dK + i * kv_part, cK + i * kv_part, kv_part, cudaMemcpyHostToDevice, s_in);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(dV + i * kv_part, cV + i * kv_part, kv_part, cudaMemcpyHostToDevice, s_in);
+        if (e == cudaSuccess && hG) e = cudaMemcpyAsync(dG + i * q_part, cG + i * q_part, q_part, cudaMemcpyHostToDevice, s_in);
+        if (e == cudaSuccess) e = cudaEventRecord(ev_in[i], s_in);
+        if (e != cudaSuccess) { cleanup(); return STILL_ERR_CUDA; }
+    }
+    for (int i = 0; i < n_parts && rc == STILL_OK; ++i) {
+        const int kv0 = (i % parts_per_b) * g;   // first KV head of the part: selects its slice of the NP-Map weights
+        if (cudaStreamWaitEvent(st, ev_in[i], 0) != cudaSuccess) { rc = STILL_ERR_CUDA; break; }
+        rc = still_hybrid_attn_fwd(&sub, N, dQ + i * q_part, dK + i * kv_part, dV + i * kv_part,
+                                   hG ? dG + i * q_part : nullptr,
+                                   hWq ? dWq + (size_t)kv0 * rep * p->d * p->d_f * es : nullptr,
+                                   hbq ? dbq + (size_t)kv0 * rep * p->d_f * es : nullptr,
+                                   hWk ? dWk + (size_t)kv0 * p->d * p->d_f * es : nullptr,
+                                   hbk ? dbk + (size_t)kv0 * p->d_f * es : nullptr, dY + i * q_part,
+                                   reinterpret_cast<float *>(dsc + i * sc_part), reinterpret_cast<int32_t *>(dsi + i * si_part),
+                                   nullptr, 0, ws, ws_bytes, cuda_stream);
+        if (rc != STILL_OK) break;
+        cudaError_t e = cudaEventRecord(ev_done[i], st);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(s_out, ev_done[i], 0);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(static_cast<char *>(hY) + i * q_part, dY + i * q_part, q_part, cudaMemcpyDeviceToHost, s_out);
+        if (e == cudaSuccess && hscores)
+            e = cudaMemcpyAsync(reinterpret_cast<char *>(hscores) + i * sc_part, dsc + i * sc_part, sc_part, cudaMemcpyDeviceToHost, s_out);
+        if (e == cudaSuccess && hsel_idx && p->topk > 0)
+            e = cudaMemcpyAsync(reinterpret_cast<char *>(hsel_idx) + i * si_part, dsi + i * si_part, si_part, cudaMemcpyDeviceToHost, s_out);
+        if (e != cudaSuccess) rc = STILL_ERR_CUDA;
+    }
+    // everything enqueued has to drain before the events go and before the host reads the outputs
+    cudaError_t e1 = cudaStreamSynchronize(s_in), e2 = cudaStreamSynchronize(st), e3 = cudaStreamSynchronize(s_out);
+    cleanup();
     if (rc != STILL_OK) return rc;
-    STILL_CUDA(cudaMemcpyAsync(hY, dY, qb, cudaMemcpyDeviceToHost, st));
-    if (hscores) STILL_CUDA(cudaMemcpyAsync(hscores, dsc, scb, cudaMemcpyDeviceToHost, st));
-    if (hsel_idx && p->topk > 0) STILL_CUDA(cudaMemcpyAsync(hsel_idx, dsi, sib, cudaMemcpyDeviceToHost, st));
-    STILL_CUDA(cudaStreamSynchronize(st));
+    if (e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess) return STILL_ERR_CUDA;
     return STILL_OK;
 }
 
