@@ -151,6 +151,38 @@ def oracle_sample(w, lam, n_heads, n_rows, seed=0):
     return total, threads, sample, t_fixed + t_rows
 
 
+def oracle_decode_sample(w, lam, n_rows=257):
+    """CPU oracle for the decode workload: the per-token cost of the softmax/merge step at the end of the
+    prefix (difference between n_rows and 1 answered rows, all prefix work excluded), one head per thread,
+    scaled to B * H heads per step."""
+    import multiprocessing
+
+    import numpy as np
+
+    from oracle import still_oracle as oracle
+    from paper_2602_02180_b200 import synth
+
+    n_heads = max(1, min(multiprocessing.cpu_count(), w.B * w.H))
+    ws = w.with_(B=1, H=n_heads, Hkv=n_heads, k=lam, N=w.N + n_rows)
+    Q, K, V = synth.make_qkv(ws, "cpu")
+    Wq, Wk = synth.make_npmap_weights(ws, "cpu")
+    f64 = lambda t: t.float().numpy().astype(np.float64)  # noqa: E731
+    Q, K, V, Wq, Wk = map(f64, (Q, K, V, Wq, Wk))
+    hp = oracle.HeadParams(w.C, lam, w.sm_scale)
+    rows = np.arange(w.N, w.N + n_rows, dtype=np.int64)
+    t0 = time.perf_counter()
+    out = oracle.layer(Q, K, V, Wq, Wk, hp, rows=rows[:1])
+    t_one = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    out = oracle.layer(Q, K, V, Wq, Wk, hp, rows=rows)
+    t_all = time.perf_counter() - t0
+    per_step_heads = max(t_all - t_one, 1e-9) / (n_rows - 1)      # n_heads heads, one token each
+    step_s = per_step_heads * (w.B * w.H) / n_heads
+    return {"value": w.B / step_s, "unit": UNIT, "cores": out["threads"], "kind": "oracle",
+            "sample": f"{n_heads} of {w.B * w.H} heads on {out['threads']} threads; softmax+merge of {n_rows} tokens after "
+                      f"the {w.N}-token prefix (prefix work excluded), scaled by head count"}
+
+
 def run_reference(args, w, lam, rank, world):
     """--impl reference: the CPU oracle as it stands, on this machine's host cores."""
     if rank != 0:
@@ -399,13 +431,44 @@ def bench_decode(args, w, lam, still, synth, torch, dist, dev, rank, world):
     roof = {"bound": "hbm", "kernel": "split-KV attend", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
             "frac": ach / peaks["hbm_gbs"], "peak_source": peaks["source"], "kernel_ms": k_ms,
             "traffic": ncu_traffic(f"attend_{w.name}_k{lam}")}
+    # end to end: every step copies that step's q, k, v from pinned host memory and reads y back
+    e2e = None
+    if not args.no_e2e:
+        hins = [tuple(x.cpu().pin_memory() for x in ins[i]) for i in range(8)]
+        dq, dk, dv = (torch.empty_like(x) for x in ins[0])
+        hy = torch.empty(w.B, w.H, w.d, dtype=w.torch_dtype).pin_memory()
+        n_e2e = min(n_steps, 64)
+        _barrier(torch, dist)
+        t0 = time.perf_counter()
+        e0.record()
+        for i in range(n_e2e):
+            hq, hk, hv = hins[i % 8]
+            dq.copy_(hq, non_blocking=True)
+            dk.copy_(hk, non_blocking=True)
+            dv.copy_(hv, non_blocking=True)
+            still.hybrid_attn_step(p, state, cap, t, dq, dk, dv, Wq, Wk, y=y)
+            hy.copy_(y, non_blocking=True)
+            torch.cuda.current_stream().synchronize()
+            t += 1
+        e1.record()
+        _barrier(torch, dist)
+        ms_e2e = max(e0.elapsed_time(e1), (time.perf_counter() - t0) * 1e3) / n_e2e
+        ms_e2e = _max_over_ranks(torch, dist, ms_e2e, dev)
+        e2e = {"value": world * w.B / (ms_e2e * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": sum(x.numel() * x.element_size() for x in hins[0]),
+               "d2h_bytes_per_step": hy.numel() * hy.element_size(), "ms_per_step": ms_e2e, "steps": n_e2e}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu = oracle_decode_sample(w, lam)
+
     return {
         "metric": "hybrid-attn decode tokens/s/layer at Llama-3-8B shape", "value": world * w.B / (ms_step * 1e-3),
         "unit": UNIT, "n_gpus": world, "steps": n_steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_step,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": w.name, "B": w.B, "H": w.H, "Hkv": w.Hkv, "d": w.d, "prefix": w.N, "chunk": w.C,
                    "topk": lam, "l2": "K/V history larger than L2 (no flush)"},
-        "clocks": clocks, "e2e": None, "gpu_launches": launches * n_steps, "roofline": roof, "cpu_baseline": None,
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches * n_steps, "roofline": roof, "cpu_baseline": cpu,
     }
 
 
