@@ -56,14 +56,27 @@ __device__ __forceinline__ void mma_ts_tf32(uint32_t d_tmem, uint32_t a_tmem, ui
 // ------------------------------------------------------------------------------------------
 // NP-Map
 // ------------------------------------------------------------------------------------------
+// Shared memory of the NP-Map kernel: the x and W tiles, later reused as the staging space of the output
+// (four warps x 32 padded rows); the region is the larger of the two.
+template <int D, int DF, typename TOut>
+struct NpmapSmem {
+    static constexpr int kHalfChunks = 32 * (int)sizeof(TOut) / 16;   // 16-byte pieces of 32 features
+    static constexpr int kStageRow = 2 * kHalfChunks * 16 + 16;       // padded: conflict-free 16-byte accesses
+    static constexpr int kTiles = 128 * D * 2 + D * DF * 2;
+    static constexpr int kStage = 4 * 32 * kStageRow;
+    static constexpr int kRegion = ((kTiles > kStage ? kTiles : kStage) + 1023) / 1024 * 1024;
+    static constexpr int kTotal = kRegion + 64;
+};
+
 template <int D, int DF, typename TOut>
 __global__ void __launch_bounds__(192, 3)
 npmap_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
                 const __nv_bfloat16 *__restrict__ bias, TOut *__restrict__ phi, int *status, int heads, int N) {
     constexpr int kXBytes = 128 * D * 2, kWBytes = D * DF * 2;
+    using Lay = NpmapSmem<D, DF, TOut>;
     extern __shared__ __align__(1024) uint8_t smem[];
     uint8_t *x_s = smem, *w_s = smem + kXBytes;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + kXBytes + kWBytes);  // [0] loads done, [1] f done
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + Lay::kRegion);  // [0] loads done, [1] f done
     uint32_t *tmem_base_slot = reinterpret_cast<uint32_t *>(bars + 2);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_base_slot + 1);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -127,6 +140,8 @@ npmap_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
                     }
                 }
         }
+        // all four epilogue warps are done reading the x tile before any of them reuses it as staging space
+        asm volatile("bar.sync 1, 128;" ::: "memory");
         if (ok) ok = mbar_wait(bars + 1, 0, abort_flag, status, 32);
         ok = __all_sync(0xffffffffu, ok);
         if (ok) {
@@ -169,45 +184,55 @@ npmap_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
                 }
             }
             const float ip = 1.f / zp, in = 1.f / zn;
-            const bool live = R0 + r < N;
-            TOut *out = phi + (row0 + r) * (2 * DF);
+            // The features leave through shared memory: a thread owns a row, but a store instruction in
+            // which every lane writes to a different row touches 32 lines; staged, 8 (fp32) or 4 (bf16)
+            // consecutive lanes write one 128- or 64-byte run of a row.  Each warp stages and writes its
+            // own 32 rows (the x / W tiles are dead by now), 32 columns of both halves at a time.
+            constexpr int kHalfChunks = Lay::kHalfChunks, kStageRow = Lay::kStageRow;
+            uint8_t *stage = smem + wq * (32 * kStageRow);
+            const int rows_live = min(32, N - (R0 + wq * 32));        // rows of this warp that exist
 #pragma unroll 1
             for (int q = 0; q < DF / 32; ++q) {
                 uint32_t v[32];
                 tmem_ld32(taddr + q * 32, v);
                 tmem_wait_ld();
-                float u[32];
+                uint8_t *mine = stage + lane * kStageRow;
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    float x = __uint_as_float(v[j]);
-                    if (bh_ != nullptr) x += __bfloat162float(bh_[q * 32 + j]);
-                    u[j] = x * ratio;
-                }
-                if (live) {
+                for (int j = 0; j < 32; j += 4) {
+                    float u[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        float x = __uint_as_float(v[j + e]);
+                        if (bh_ != nullptr) x += __bfloat162float(bh_[q * 32 + j + e]);
+                        u[e] = x * ratio;
+                    }
                     if constexpr (sizeof(TOut) == 4) {
-#pragma unroll
-                        for (int j = 0; j < 32; j += 4) {
-                            *reinterpret_cast<float4 *>(out + q * 32 + j) =
-                                make_float4(ex2(u[j] - umax) * ip, ex2(u[j + 1] - umax) * ip, ex2(u[j + 2] - umax) * ip,
-                                            ex2(u[j + 3] - umax) * ip);
-                            *reinterpret_cast<float4 *>(out + DF + q * 32 + j) =
-                                make_float4(ex2(umin - u[j]) * in, ex2(umin - u[j + 1]) * in, ex2(umin - u[j + 2]) * in,
-                                            ex2(umin - u[j + 3]) * in);
-                        }
+                        *reinterpret_cast<float4 *>(mine + j * 4) =
+                            make_float4(ex2(u[0] - umax) * ip, ex2(u[1] - umax) * ip, ex2(u[2] - umax) * ip, ex2(u[3] - umax) * ip);
+                        *reinterpret_cast<float4 *>(mine + kHalfChunks * 16 + j * 4) =
+                            make_float4(ex2(umin - u[0]) * in, ex2(umin - u[1]) * in, ex2(umin - u[2]) * in, ex2(umin - u[3]) * in);
                     } else {
-#pragma unroll
-                        for (int j = 0; j < 32; j += 8) {
-                            uint32_t pp[4], nn[4];
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                pp[e] = pack_bf16(ex2(u[j + 2 * e] - umax) * ip, ex2(u[j + 2 * e + 1] - umax) * ip);
-                                nn[e] = pack_bf16(ex2(umin - u[j + 2 * e]) * in, ex2(umin - u[j + 2 * e + 1]) * in);
-                            }
-                            *reinterpret_cast<uint4 *>(out + q * 32 + j) = make_uint4(pp[0], pp[1], pp[2], pp[3]);
-                            *reinterpret_cast<uint4 *>(out + DF + q * 32 + j) = make_uint4(nn[0], nn[1], nn[2], nn[3]);
-                        }
+                        *reinterpret_cast<uint2 *>(mine + j * 2) =
+                            make_uint2(pack_bf16(ex2(u[0] - umax) * ip, ex2(u[1] - umax) * ip),
+                                       pack_bf16(ex2(u[2] - umax) * ip, ex2(u[3] - umax) * ip));
+                        *reinterpret_cast<uint2 *>(mine + kHalfChunks * 16 + j * 2) =
+                            make_uint2(pack_bf16(ex2(umin - u[0]) * in, ex2(umin - u[1]) * in),
+                                       pack_bf16(ex2(umin - u[2]) * in, ex2(umin - u[3]) * in));
                     }
                 }
+                __syncwarp();
+#pragma unroll
+                for (int it = 0; it < 2 * kHalfChunks; ++it) {
+                    const int id = it * 32 + lane, row = id / (2 * kHalfChunks), c = id % (2 * kHalfChunks);
+                    if (row < rows_live) {
+                        const uint4 val = *reinterpret_cast<const uint4 *>(stage + row * kStageRow + c * 16);
+                        uint8_t *dst = reinterpret_cast<uint8_t *>(phi + (row0 + wq * 32 + row) * (2 * DF) +
+                                                                   (c < kHalfChunks ? 0 : DF) + q * 32) +
+                                       (c % kHalfChunks) * 16;
+                        *reinterpret_cast<uint4 *>(dst) = val;
+                    }
+                }
+                __syncwarp();
             }
         }
     }
@@ -514,7 +539,7 @@ int launch_npmap(const void *X, const void *W, const void *bias, void *phi, int 
     if (!make_map_2d(&tx, X, (unsigned long long)B * heads * N, D, 128, false) ||
         !make_map_2d(&tw, W, (unsigned long long)heads * D, DF, D, false))
         return STILL_ERR_CUDA;
-    constexpr int kSmem = 128 * D * 2 + D * DF * 2 + 64;
+    constexpr int kSmem = NpmapSmem<D, DF, TOut>::kTotal;
     if (cudaFuncSetAttribute(npmap_tc_kernel<D, DF, TOut>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) !=
         cudaSuccess)
         return STILL_ERR_CUDA;
