@@ -463,30 +463,47 @@ la_scan_tc_kernel(const __grid_constant__ CUtensorMap tm_phik, const __grid_cons
                 for (int j = 0; j < sc && nu < n_upd; ++j) mask_tile();
             if (ok) ok = mbar_wait(r_done + (nq & 1), (nq >> 1) & 1, abort_flag, status, 45);
             ok = __all_sync(0xffffffffu, ok);
+            // The result leaves through shared memory (the phi(Q) stage this read-out has just consumed is free
+            // until the workers release it): a thread holds one value column of 64 tokens, but the rows of
+            // N_LA are token-major, and a column-wise store loop costs over a hundred clocks per instruction.
+            float *stg = reinterpret_cast<float *>(smem + P::kQ + (nq & 1) * P::kPhiQ);   // [64 tokens][64 columns], then D_LA [64]
+            const int base = u * 64;
             if (ok) {
                 tc_fence_after();
                 uint32_t o[64];
                 tmem_ld32(taddr + col_out + (nq & 1) * 64, o);
                 tmem_ld32(taddr + col_out + (nq & 1) * 64 + 32, o + 32);
                 tmem_wait_ld();
-                const int base = u * 64;
-                if (e < 64) {
-                    const long long off = ((long long)bh * N + base) * d + e0 + e;
-#pragma unroll
-                    for (int t = 0; t < 64; ++t)
-                        if (base + t < N) {
-                            float v = __uint_as_float(o[t]);
-                            if (G != nullptr) v *= __bfloat162float(G[off + (long long)t * d]);
-                            N_LA[off + (long long)t * d] = v;
-                        }
-                } else if (e == 64 && blockIdx.y == 0) {
-#pragma unroll
-                    for (int t = 0; t < 64; ++t)
-                        if (base + t < N) D_LA[(long long)bh * N + base + t] = __uint_as_float(o[t]);
-                }
                 tc_fence_before();
+                if (e < 64) {
+#pragma unroll
+                    for (int t = 0; t < 64; ++t) stg[t * 64 + e] = __uint_as_float(o[t]);
+                } else if (e == 64) {
+#pragma unroll
+                    for (int t = 0; t < 64; ++t) stg[64 * 64 + t] = __uint_as_float(o[t]);
+                }
             }
-            __syncwarp();
+            asm volatile("bar.sync 2, 128;" ::: "memory");   // the four worker warps (always, whatever `ok`)
+            if (ok) {
+#pragma unroll
+                for (int it = 0; it < 8; ++it) {
+                    const int id = it * 128 + tid, t = id >> 4, c = id & 15;
+                    if (base + t < N) {
+                        float4 v = *reinterpret_cast<const float4 *>(stg + t * 64 + c * 4);
+                        const long long off = ((long long)bh * N + base + t) * d + e0 + c * 4;
+                        if (G != nullptr) {
+                            const uint2 gg = *reinterpret_cast<const uint2 *>(G + off);
+                            v.x *= __uint_as_float(gg.x << 16);
+                            v.y *= __uint_as_float(gg.x & 0xffff0000u);
+                            v.z *= __uint_as_float(gg.y << 16);
+                            v.w *= __uint_as_float(gg.y & 0xffff0000u);
+                        }
+                        *reinterpret_cast<float4 *>(N_LA + off) = v;
+                    }
+                }
+                if (blockIdx.y == 0 && tid < 64 && base + tid < N) D_LA[(long long)bh * N + base + tid] = stg[64 * 64 + tid];
+            }
+            asm volatile("bar.sync 2, 128;" ::: "memory");   // staging space read by all before the stage is released
             if (lane == 0) {
                 mbar_arrive(out_free + (nq & 1));
                 mbar_arrive(q_empty + (nq & 1));
