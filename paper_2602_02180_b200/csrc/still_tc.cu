@@ -422,10 +422,18 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 ++n_seen;
             }
             // ---- epilogue: y = (O e^{m-ms} + e^{-ms} N_LA) / (l e^{m-ms} + e^{-ms} D_LA), ms = max(m, 0)
+            // A thread owns a row, but loads / stores in which every lane touches a different row cost a
+            // memory instruction per 16 bytes and row; so N_LA comes in and Y goes out through shared memory
+            // with 16 consecutive lanes per row.  The staging space is this warp's 32 rows of the tile's Q
+            // region (one row = D bf16 = 2 D bytes), free once the tile's last Q K^T has completed; 16-byte
+            // pieces are swizzled by the row so that row-wise and piece-wise accesses avoid bank conflicts.
             if (ok) ok = mbar_wait(o_final + x, 0, abort_flag, status, 9);
+            ok = __all_sync(0xffffffffu, ok);
             if (ok) {
                 tc_fence_after();
-                const long long row_off = ((long long)bh * N + t) * D;
+                constexpr int kRowBytes = D * 2, kPieces = kRowBytes / 16;   // pieces of 16 bytes per staged row
+                uint8_t *stg = smem + P::kQ + x * P::kTileBytes + (warp & 3) * 32 * kRowBytes;
+                const int t0 = R0 + x * kBlockM + (warp & 3) * 32;           // first row of this warp
                 float fs = 1.f, fl = 0.f, dla = 0.f;
                 if (D_LA != nullptr && t < N) {
                     dla = D_LA[(long long)bh * N + t];
@@ -437,27 +445,54 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     }
                 }
                 const float inv = 1.f / (l_sum * fs + fl * dla);
+                const bool with_la = (D_LA != nullptr) && __any_sync(0xffffffffu, dla > 0.f);
+                uint32_t out[D / 2];   // the row as packed bf16
 #pragma unroll
-                for (int q = 0; q < D / 32; ++q) {
-                    uint32_t orow[32];
-                    tmem_ld32(lane_addr + col_o(x) + q * 32, orow);
-                    tmem_wait_ld();
-                    if (t < N) {
-                        uint32_t out[16];
+                for (int hh = 0; hh < 2; ++hh) {   // halves of D / 2 columns: as fp32 they fill one staged row
+                    if (with_la) {
+                        __syncwarp();
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            float a0 = __uint_as_float(orow[2 * j]) * fs, a1 = __uint_as_float(orow[2 * j + 1]) * fs;
-                            if (dla > 0.f) {
-                                const float2 nl = *reinterpret_cast<const float2 *>(N_LA + row_off + q * 32 + 2 * j);
-                                a0 += fl * nl.x;
-                                a1 += fl * nl.y;
-                            }
-                            out[j] = pack_bf16(a0 * inv, a1 * inv);
+                        for (int it = 0; it < kPieces; ++it) {
+                            const int id = it * 32 + lane, row = id / kPieces, c = id % kPieces;
+                            uint4 v = make_uint4(0, 0, 0, 0);
+                            if (t0 + row < N)
+                                v = *reinterpret_cast<const uint4 *>(N_LA + ((long long)bh * N + t0 + row) * D + hh * (D / 2) + c * 4);
+                            *reinterpret_cast<uint4 *>(stg + row * kRowBytes + ((c ^ (row & (kPieces - 1))) << 4)) = v;
                         }
-                        uint4 *dst = reinterpret_cast<uint4 *>(Y + row_off + q * 32);
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) dst[j] = make_uint4(out[4 * j], out[4 * j + 1], out[4 * j + 2], out[4 * j + 3]);
+                        __syncwarp();
                     }
+#pragma unroll
+                    for (int q = 0; q < D / 64; ++q) {
+                        uint32_t orow[32];
+                        tmem_ld32(lane_addr + col_o(x) + hh * (D / 2) + q * 32, orow);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int j4 = 0; j4 < 8; ++j4) {
+                            float4 nl = make_float4(0.f, 0.f, 0.f, 0.f);
+                            if (with_la)
+                                nl = *reinterpret_cast<const float4 *>(stg + lane * kRowBytes + (((q * 8 + j4) ^ (lane & (kPieces - 1))) << 4));
+                            const float a0 = fmaf(fl, nl.x, __uint_as_float(orow[4 * j4]) * fs);
+                            const float a1 = fmaf(fl, nl.y, __uint_as_float(orow[4 * j4 + 1]) * fs);
+                            const float a2 = fmaf(fl, nl.z, __uint_as_float(orow[4 * j4 + 2]) * fs);
+                            const float a3 = fmaf(fl, nl.w, __uint_as_float(orow[4 * j4 + 3]) * fs);
+                            out[hh * (D / 4) + q * 16 + 2 * j4] = pack_bf16(a0 * inv, a1 * inv);
+                            out[hh * (D / 4) + q * 16 + 2 * j4 + 1] = pack_bf16(a2 * inv, a3 * inv);
+                        }
+                    }
+                }
+                // Y: own row into the staging space, then the warp writes its 32 rows piece-wise
+                __syncwarp();
+#pragma unroll
+                for (int c = 0; c < kPieces; ++c)
+                    *reinterpret_cast<uint4 *>(stg + lane * kRowBytes + ((c ^ (lane & (kPieces - 1))) << 4)) =
+                        make_uint4(out[4 * c], out[4 * c + 1], out[4 * c + 2], out[4 * c + 3]);
+                __syncwarp();
+#pragma unroll
+                for (int it = 0; it < kPieces; ++it) {
+                    const int id = it * 32 + lane, row = id / kPieces, c = id % kPieces;
+                    if (t0 + row < N)
+                        *reinterpret_cast<uint4 *>(Y + ((long long)bh * N + t0 + row) * D + c * 8) =
+                            *reinterpret_cast<const uint4 *>(stg + row * kRowBytes + ((c ^ (row & (kPieces - 1))) << 4));
                 }
             }
         }
