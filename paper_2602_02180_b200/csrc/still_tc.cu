@@ -578,57 +578,107 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         const int wq = warp & 3;                       // TMEM lane quarter this warp may read
         const int r = wq * 32 + lane, t = R0 + r;
         const uint32_t taddr = tmem_base + ((uint32_t)(wq * 32) << 16) + (uint32_t)(wq * 32 + kBlockN - C);
-        constexpr int kChunks = (C + 32) / 32;
         const bool ok = mbar_wait(bars + 1, 0, abort_flag, status, 21);
         tc_fence_after();
         float score = 0.f;
         if (ok) {
-            // element j of the warp's C+32 columns is the key at position R0 + 32 wq - C + j
-            const int pos0 = R0 + wq * 32 - C;
-            float mx = -INFINITY;
-#pragma unroll 1
-            for (int q = 0; q < kChunks; ++q) {
-                uint32_t v[32];
+            // Element j of the warp's C+32 columns is the key at position R0 + 32 wq - C + j, and the window of
+            // the row in lane l is j in [l+1, l+C].  Columns [32, C) lie in every lane's window; of columns jj
+            // and C + jj (jj < 32) exactly one does (the first if jj > l).  So the first and the last block of
+            // 32 columns fold into one, and a row becomes C values without gaps: block 0 is the folded one (the
+            // token itself sits at jj = l), blocks 1 .. C/32-1 are columns [32 q, 32 q + 32).  Keys at negative
+            // positions (first tile of a sequence only) are set to -inf, which the exponential turns into 0.
+            constexpr int kBlocks = C / 32;
+            const bool first_tile = R0 == 0;
+            auto load_block = [&](int q, uint32_t (&v)[32]) {
                 tmem_ld32(taddr + q * 32, v);
-                tmem_wait_ld();
+                if (q == 0) {
+                    uint32_t w[32];
+                    tmem_ld32(taddr + C, w);
+                    tmem_wait_ld();
 #pragma unroll
-                for (int jj = 0; jj < 32; ++jj) {
-                    const int j = q * 32 + jj;
-                    const bool valid = (j > lane) && (j <= lane + C) && (pos0 + j >= 0);
-                    if (valid) mx = fmaxf(mx, __uint_as_float(v[jj]));
+                    for (int jj = 0; jj < 32; ++jj) v[jj] = (jj > lane) ? v[jj] : w[jj];
+                } else {
+                    tmem_wait_ld();
                 }
-            }
-            const float neg_m = -mx * scale_log2;
-            float z_all = 0.f, z_nd = 0.f;
-#pragma unroll 1
-            for (int q = 0; q < kChunks; ++q) {
-                uint32_t v[32];
-                tmem_ld32(taddr + q * 32, v);
-                tmem_wait_ld();
+                if (first_tile) {
+                    const int n_neg = C - wq * 32;   // columns below n_neg are before the start of the sequence
 #pragma unroll
-                for (int jj = 0; jj < 32; ++jj) {
-                    const int j = q * 32 + jj;
-                    const bool valid = (j > lane) && (j <= lane + C) && (pos0 + j >= 0);
-                    const float e = valid ? ex2(fmaf(__uint_as_float(v[jj]), scale_log2, neg_m)) : 0.f;
-                    z_all += e;
-                    if (j != lane + C) z_nd += e;
+                    for (int jj = 0; jj < 32; ++jj)
+                        if (q * 32 + jj < n_neg && (q > 0 || jj > lane)) v[jj] = 0xff800000u;
                 }
-            }
-            const float inv_all = 1.f / z_all, inv_nd = z_nd > 0.f ? 1.f / z_nd : 0.f;
-#pragma unroll 1
-            for (int q = 0; q < kChunks; ++q) {
-                uint32_t v[32];
-                tmem_ld32(taddr + q * 32, v);
-                tmem_wait_ld();
+            };
+            if constexpr (kBlocks == 2) {
+                // the row fits the register file: one read of tensor memory, exponentials kept in place
+                uint32_t v0[32], v1[32];
+                load_block(0, v0);
+                load_block(1, v1);
+                float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+                for (int jj = 0; jj < 32; jj += 2) {
+                    mx0 = max3(mx0, __uint_as_float(v0[jj]), __uint_as_float(v0[jj + 1]));
+                    mx1 = max3(mx1, __uint_as_float(v1[jj]), __uint_as_float(v1[jj + 1]));
+                }
+                const float neg_m = -fmaxf(mx0, mx1) * scale_log2;
+                float z0 = 0.f, z1 = 0.f, e_self = 0.f;
 #pragma unroll
                 for (int jj = 0; jj < 32; ++jj) {
-                    const int j = q * 32 + jj;
-                    const bool valid = (j > lane) && (j <= lane + C) && (pos0 + j >= 0);
-                    const float e = valid ? ex2(fmaf(__uint_as_float(v[jj]), scale_log2, neg_m)) : 0.f;
-                    const float a = e * inv_all;
-                    const float bb = (j != lane + C) ? e * inv_nd : 0.f;
-                    // a * ln((a + eps) / (bb + eps)); an invalid element has a = 0 and adds nothing
-                    score += a * (__log2f(a + eps) - __log2f(bb + eps));
+                    const float e0 = ex2(fmaf(__uint_as_float(v0[jj]), scale_log2, neg_m));
+                    const float e1 = ex2(fmaf(__uint_as_float(v1[jj]), scale_log2, neg_m));
+                    v1[jj] = __float_as_uint(e1);
+                    z1 += e1;
+                    if (jj == lane) e_self = e0;
+                    else z0 += e0;                    // the sum without the token itself is formed directly
+                    v0[jj] = __float_as_uint(e0);
+                }
+                const float z_nd = z0 + z1, z_all = z_nd + e_self;
+                const float inv_all = 1.f / z_all, inv_nd = z_nd > 0.f ? 1.f / z_nd : 0.f;
+                float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+                for (int jj = 0; jj < 32; ++jj) {
+                    // a * ln((a + eps) / (b + eps)); a masked key has a = b = 0 and adds nothing
+                    const float e0 = __uint_as_float(v0[jj]), e1 = __uint_as_float(v1[jj]);
+                    const float a0 = e0 * inv_all, a1 = e1 * inv_all;
+                    const float b0 = (jj == lane) ? 0.f : e0 * inv_nd, b1 = e1 * inv_nd;
+                    s0 += a0 * (__log2f(a0 + eps) - __log2f(b0 + eps));
+                    s1 += a1 * (__log2f(a1 + eps) - __log2f(b1 + eps));
+                }
+                score = s0 + s1;
+            } else {
+                float mx = -INFINITY;
+#pragma unroll 1
+                for (int q = 0; q < kBlocks; ++q) {
+                    uint32_t v[32];
+                    load_block(q, v);
+#pragma unroll
+                    for (int jj = 0; jj < 32; jj += 2) mx = max3(mx, __uint_as_float(v[jj]), __uint_as_float(v[jj + 1]));
+                }
+                const float neg_m = -mx * scale_log2;
+                float z_nd = 0.f, e_self = 0.f;
+#pragma unroll 1
+                for (int q = 0; q < kBlocks; ++q) {
+                    uint32_t v[32];
+                    load_block(q, v);
+#pragma unroll
+                    for (int jj = 0; jj < 32; ++jj) {
+                        const float e = ex2(fmaf(__uint_as_float(v[jj]), scale_log2, neg_m));
+                        if (q == 0 && jj == lane) e_self = e;
+                        else z_nd += e;
+                    }
+                }
+                const float z_all = z_nd + e_self;
+                const float inv_all = 1.f / z_all, inv_nd = z_nd > 0.f ? 1.f / z_nd : 0.f;
+#pragma unroll 1
+                for (int q = 0; q < kBlocks; ++q) {
+                    uint32_t v[32];
+                    load_block(q, v);
+#pragma unroll
+                    for (int jj = 0; jj < 32; ++jj) {
+                        const float e = ex2(fmaf(__uint_as_float(v[jj]), scale_log2, neg_m));
+                        const float a = e * inv_all;
+                        const float bb = (q == 0 && jj == lane) ? 0.f : e * inv_nd;
+                        score += a * (__log2f(a + eps) - __log2f(bb + eps));
+                    }
                 }
             }
             score *= 0.6931471805599453f;
