@@ -178,11 +178,13 @@ int still_hybrid_attn_step(const still_params_t *p, void *state, int64_t state_m
  * still_hybrid_attn_fwd and copies Y (and scores / sel_idx when not NULL) back.
  * `arena` is device memory of at least still_host_arena_bytes(p, N) bytes; it
  * holds the staged tensors and the workspace.  The (batch, KV-head group) units
- * are independent, so the call is cut into up to eight parts whose host-to-device
- * copies, compute and device-to-host copies overlap (two side streams created
- * on first use per host thread, ordered after the work already enqueued on
- * `cuda_stream`).  The call returns after synchronising all of them, so the host
- * outputs are valid on return.
+ * are independent, so the call is cut into up to sixteen parts whose host-to-device
+ * copies, compute and device-to-host copies overlap; the parts compute alternately
+ * on `cuda_stream` and on a second stream, so that one part's last thread blocks
+ * run beside the next part's first ones (three side streams created on first use
+ * per host thread, ordered after the work already enqueued on `cuda_stream`).  The
+ * call returns after synchronising all of them, so the host outputs are valid on
+ * return.
  */
 size_t still_host_arena_bytes(const still_params_t *p, int64_t N);
 int still_hybrid_attn_fwd_host(const still_params_t *p, int64_t N, const void *hQ, const void *hK,

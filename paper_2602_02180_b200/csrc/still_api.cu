@@ -479,18 +479,22 @@ int still_hybrid_attn_fwd_host(const still_params_t *p, int64_t N, const void *h
     if (hWk) STILL_CUDA(cudaMemcpyAsync(dWk, hWk, wkb, cudaMemcpyHostToDevice, st));
     if (hbk) STILL_CUDA(cudaMemcpyAsync(dbk, hbk, bkb, cudaMemcpyHostToDevice, st));
 
-    // The (batch, KV-head group) units are independent, so the call is cut into up to eight parts --
+    // The (batch, KV-head group) units are independent, so the call is cut into up to sixteen parts --
     // contiguous ranges of KV heads of one batch entry with their query heads -- and pipelined: the
     // host-to-device copies of part i+1 and the device-to-host copies of part i-1 run on two side
-    // streams while part i computes on the caller's stream (PCIe is full duplex, and the copies are as
-    // long as the compute at the benchmark shapes).
-    static thread_local cudaStream_t s_in = nullptr, s_out = nullptr;
+    // streams while part i computes (PCIe is full duplex, and the copies are as long as the compute at
+    // the benchmark shapes).  What the pipeline cannot hide is the first part's copy in and the last
+    // part's copy out, hence small parts; and since a small part's kernels end in a partly filled wave,
+    // the parts compute alternately on the caller's stream and on a second one, each with its own
+    // workspace, so that the next part's thread blocks fill that tail.
+    static thread_local cudaStream_t s_in = nullptr, s_out = nullptr, s_alt = nullptr;
     if (!s_in) {
         STILL_CUDA(cudaStreamCreateWithFlags(&s_in, cudaStreamNonBlocking));
         STILL_CUDA(cudaStreamCreateWithFlags(&s_out, cudaStreamNonBlocking));
+        STILL_CUDA(cudaStreamCreateWithFlags(&s_alt, cudaStreamNonBlocking));
     }
     const int rep = p->H / p->Hkv;
-    int g = std::max(1, p->Hkv * p->B / 8);          // KV heads per part
+    int g = std::max(1, p->Hkv * p->B / 16);         // KV heads per part
     while (p->Hkv % g != 0) --g;
     const int parts_per_b = p->Hkv / g, n_parts = p->B * parts_per_b;
     constexpr int kMaxParts = 64;
@@ -528,10 +532,14 @@ int still_hybrid_attn_fwd_host(const still_params_t *p, int64_t N, const void *h
     // the side streams start after what the caller has already enqueued (and after the weights)
     STILL_CUDA(cudaEventRecord(ev_start, st));
     STILL_CUDA(cudaStreamWaitEvent(s_in, ev_start, 0));
+    STILL_CUDA(cudaStreamWaitEvent(s_alt, ev_start, 0));
     still_params_t sub = *p;
     sub.B = 1;
     sub.Hkv = g;
     sub.H = g * rep;
+    // a second workspace for the alternate compute stream, if the arena's workspace holds two of a part's size
+    const size_t ws_part = align_up(plan_fwd(&sub, N).total, 1024);
+    const bool two_streams = n_parts > 1 && 2 * ws_part <= ws_bytes;
     const size_t q_part = (size_t)g * rep * N * p->d * es, kv_part = (size_t)g * N * p->d * es;
     const size_t sc_part = (size_t)g * rep * N * 4, si_part = (size_t)g * rep * T * std::max(p->topk, 1) * 4;
     const char *cQ = static_cast<const char *>(hQ), *cK = static_cast<const char *>(hK), *cV = static_cast<const char *>(hV);
@@ -546,7 +554,11 @@ int still_hybrid_attn_fwd_host(const still_params_t *p, int64_t N, const void *h
     }
     for (int i = 0; i < n_parts && rc == STILL_OK; ++i) {
         const int kv0 = (i % parts_per_b) * g;   // first KV head of the part: selects its slice of the NP-Map weights
-        if (cudaStreamWaitEvent(st, ev_in[i], 0) != cudaSuccess) { rc = STILL_ERR_CUDA; break; }
+        const bool alt = two_streams && (i & 1);
+        cudaStream_t cs = alt ? s_alt : st;
+        char *ws_i = alt ? ws + ws_part : ws;
+        const size_t ws_i_bytes = two_streams ? ws_part : ws_bytes;
+        if (cudaStreamWaitEvent(cs, ev_in[i], 0) != cudaSuccess) { rc = STILL_ERR_CUDA; break; }
         rc = still_hybrid_attn_fwd(&sub, N, dQ + i * q_part, dK + i * kv_part, dV + i * kv_part,
                                    hG ? dG + i * q_part : nullptr,
                                    hWq ? dWq + (size_t)kv0 * rep * p->d * p->d_f * es : nullptr,
@@ -554,9 +566,9 @@ int still_hybrid_attn_fwd_host(const still_params_t *p, int64_t N, const void *h
                                    hWk ? dWk + (size_t)kv0 * p->d * p->d_f * es : nullptr,
                                    hbk ? dbk + (size_t)kv0 * p->d_f * es : nullptr, dY + i * q_part,
                                    reinterpret_cast<float *>(dsc + i * sc_part), reinterpret_cast<int32_t *>(dsi + i * si_part),
-                                   nullptr, 0, ws, ws_bytes, cuda_stream);
+                                   nullptr, 0, ws_i, ws_i_bytes, cs);
         if (rc != STILL_OK) break;
-        cudaError_t e = cudaEventRecord(ev_done[i], st);
+        cudaError_t e = cudaEventRecord(ev_done[i], cs);
         if (e == cudaSuccess) e = cudaStreamWaitEvent(s_out, ev_done[i], 0);
         if (e == cudaSuccess) e = cudaMemcpyAsync(static_cast<char *>(hY) + i * q_part, dY + i * q_part, q_part, cudaMemcpyDeviceToHost, s_out);
         if (e == cudaSuccess && hscores)
@@ -566,10 +578,11 @@ int still_hybrid_attn_fwd_host(const still_params_t *p, int64_t N, const void *h
         if (e != cudaSuccess) rc = STILL_ERR_CUDA;
     }
     // everything enqueued has to drain before the events go and before the host reads the outputs
-    cudaError_t e1 = cudaStreamSynchronize(s_in), e2 = cudaStreamSynchronize(st), e3 = cudaStreamSynchronize(s_out);
+    cudaError_t e1 = cudaStreamSynchronize(s_in), e2 = cudaStreamSynchronize(st), e3 = cudaStreamSynchronize(s_alt);
+    cudaError_t e4 = cudaStreamSynchronize(s_out);
     cleanup();
     if (rc != STILL_OK) return rc;
-    if (e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess) return STILL_ERR_CUDA;
+    if (e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess || e4 != cudaSuccess) return STILL_ERR_CUDA;
     return STILL_OK;
 }
 
