@@ -81,6 +81,29 @@ def test_paper_literal_scale_one():
         assert np.abs(U.f64(Y[b, h]) - out["y"]).max() < 1e-4
 
 
+@pytest.mark.parametrize("k", [64, 16])
+def test_growing_logits_rescale_the_accumulator(k):
+    # The tensor-core kernel keeps a row's softmax reference until a tile's maximum exceeds it by 2^8 and then
+    # rescales the output accumulator.  Logits that grow by ~7 nats per 128-key tile, plus one key far above the
+    # rest in the second half of a tile, make that happen in every tile and in both halves.
+    w = _small("t", "bf16", 1, 4, 2, 128, 128 * 7 + 40, 64, k)
+    Q, K, V = synth.make_qkv(w, "cuda")
+    t = torch.arange(w.N, device="cuda")
+    Q = Q.float()
+    K = K.float()
+    Q[..., 0] += 8.0
+    K[..., 0] += (10.0 * (t // 128)).view(1, 1, -1)
+    K[:, :, 128 * 3 + 100, 0] += 60.0
+    Q, K = Q.to(torch.bfloat16), K.to(torch.bfloat16)
+    Wq, Wk = synth.make_npmap_weights(w, "cuda")
+    Y, scores, sel = still.hybrid_attn_fwd(U.params_of(w), Q, K, V, Wq, Wk)
+    torch.cuda.synchronize()
+    assert torch.isfinite(Y.float()).all()
+    heads = U.sample_heads(w, 4)
+    U.check_selection(scores, sel, w.C, w.k, heads)
+    U.check_outputs(w, Q, K, V, Wq, Wk, Y, scores, sel, heads)
+
+
 def test_run_to_run_determinism():
     w = _small("t", "bf16", 1, 4, 2, 64, 500, 64, 16)
     a = U.run_prefill(w)
