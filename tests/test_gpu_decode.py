@@ -12,13 +12,15 @@ from tests import util_parity as U
 pytestmark = pytest.mark.gpu
 
 
-def _decode_case(w, n0, n_steps, gate=False):
+def _decode_case(w, n0, n_steps, gate=False, tweak=None):
     """Prefill n0 tokens into a state, decode n_steps more, compare every decoded row with
     the oracle's chunk-wise form over the whole sequence (the GPU's selection forced)."""
     dev = "cuda"
     N = n0 + n_steps
     wN = w.with_(N=N)
     Q, K, V = synth.make_qkv(wN, dev)
+    if tweak is not None:
+        Q, K, V = tweak(Q, K, V)
     Wq, Wk = synth.make_npmap_weights(wN, dev)
     G = synth.make_gate(wN, dev) if gate else None
     p = U.params_of(w)
@@ -91,6 +93,22 @@ def _decode_case(w, n0, n_steps, gate=False):
 def test_decode_matches_oracle(dtype, B, H, Hkv, d, C, k, n0, steps):
     w = synth.Workload("t", B, H, Hkv, d, n0, C, k, dtype, "iid", 999)
     _decode_case(w, n0, steps, gate=(k not in (0, C)))
+
+
+@pytest.mark.parametrize("k", [64, 16])
+def test_decode_with_growing_logits(k):
+    # Logits that grow by ~7 nats per 128 tokens and one dominant key: the partial results of the key splits
+    # differ by many orders of magnitude and the merge has to bring them to one reference.
+    def tweak(Q, K, V):
+        t = torch.arange(Q.shape[2], device=Q.device)
+        Q, K = Q.float(), K.float()
+        Q[..., 0] += 8.0
+        K[..., 0] += (10.0 * (t // 128)).view(1, 1, -1)
+        K[:, :, 128 * 3 + 100, 0] += 60.0
+        return Q.to(torch.bfloat16), K.to(torch.bfloat16), V
+
+    w = synth.Workload("t", 2, 4, 2, 128, 0, 64, k, "bf16", "iid", 77)
+    _decode_case(w, 128 * 5 + 9, 70, tweak=tweak)
 
 
 def test_c5_full_size_sampled():
