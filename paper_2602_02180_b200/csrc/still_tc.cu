@@ -516,36 +516,52 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 // (element lane+C is the token itself).  With e_j = exp(l_j - max), Z = sum e_j,
 // Z' = sum_{j != t} e_j:  a_diag_j = e_j / Z,  a_nodiag_j = e_j / Z' (0 at j = t),
 // Score = sum_j a_diag_j log((a_diag_j + eps) / (a_nodiag_j + eps)).
-// Warps: 0 TMA producer, 1 MMA issuer, 2-5 score (TMEM lane quarter = warp % 4).
+// The kernel is persistent: a CTA (one per SM) walks over tiles n = blockIdx.x, blockIdx.x + gridDim.x, ...
+// (tile n = head n / n_row_blocks, rows 128 (n % n_row_blocks) ...) with two stages of shared memory and two
+// TMEM accumulators, so that the loads of tile n+1 and its UMMA run under the row epilogue of tile n.
+// Warps: 0 TMA producer, 1 MMA issuer, 2-5 score group 0 (even tiles of the CTA), 6-9 score group 1 (odd
+// tiles); TMEM lane quarter = warp % 4.
 // ---------------------------------------------------------------------------
+template <int D>
+struct ScoreSmem {
+    static constexpr int kQBytes = kBlockM * D * 2, kKBytes = 2 * kBlockN * D * 2;
+    static constexpr int kStage = kQBytes + kKBytes;
+    static constexpr int kBar = 2 * kStage;          // full[2], mma_done[2], smem_free[2], tmem_free[2]
+    static constexpr int kMisc = kBar + 8 * 8;       // tmem base, abort flag
+    static constexpr int kSc = kMisc + 16;           // [2][128] scores of the group's tile (16-byte aligned)
+    static constexpr int kBallot = kSc + 2 * kBlockM * 4;   // [2][4]
+    static constexpr int kTotal = kBallot + 2 * 4 * 4;
+    static constexpr int kAlloc = kTotal + 1024;     // slack to align the base to 1024
+};
+
 template <int D, int C>
-__global__ void __launch_bounds__(192, 2)
+__global__ void __launch_bounds__(320, 1)
 score_select_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                        float *__restrict__ scores, int32_t *__restrict__ sel_idx, int *status, int H, int Hkv,
-                       int N, int lam, float scale_log2, float eps) {
-    constexpr int kQBytes = kBlockM * D * 2, kKBytes = 2 * kBlockN * D * 2;
+                       int N, int lam, float scale_log2, float eps, int n_row_blocks, int n_tiles) {
+    using P = ScoreSmem<D>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint8_t *q_s = smem, *k_s = smem + kQBytes;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + kQBytes + kKBytes);  // [0] loads done, [1] logits done
-    uint32_t *tmem_base_slot = reinterpret_cast<uint32_t *>(bars + 2);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_base_slot + 1);
-    float *sc = reinterpret_cast<float *>(tmem_base_slot + 2);                // [128]
-    int *flag = reinterpret_cast<int *>(sc + kBlockM);                         // [128]
+    uint64_t *full = reinterpret_cast<uint64_t *>(smem + P::kBar);
+    uint64_t *mma_done = full + 2, *smem_free = full + 4, *tmem_free = full + 6;
+    uint32_t *tmem_base_slot = reinterpret_cast<uint32_t *>(smem + P::kMisc);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + P::kMisc + 8);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int bh = blockIdx.y, b = bh / H, h = bh % H, kvh = h / (H / Hkv);
-    const int R0 = blockIdx.x * kBlockM;
     const int Tn = (N + C - 1) / C;
 
     if (threadIdx.x == 0) {
-        mbar_init(bars, 1);
-        mbar_init(bars + 1, 1);
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(full + s, 1);
+            mbar_init(mma_done + s, 1);
+            mbar_init(smem_free + s, 1);
+            mbar_init(tmem_free + s, 4);   // one arrival per warp of the score group
+        }
         *abort_flag = 0;
         fence_barrier_init();
     }
     if (warp == 1) {
-        tmem_alloc(tmem_base_slot, 256);
+        tmem_alloc(tmem_base_slot, 512);
         tmem_relinquish();
     }
     tc_fence_before();
@@ -553,175 +569,228 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     tc_fence_after();
     const uint32_t tmem_base = *tmem_base_slot;
 
-    if (warp == 0 && lane == 0) {
-        mbar_expect_tx(bars, kQBytes + kKBytes);
-        const int k_row = (b * Hkv + kvh) * N + R0 - kBlockN;  // may be negative or cross into the previous head: masked by position
-        for (int half = 0; half < D / 64; ++half) {
-            tma_load_2d(q_s + half * (kBlockM * 128), &tm_q, bars, half * 64, bh * N + R0);
-            // K-major operand of 256 rows: per 64-column half, rows 0..255 contiguous
-            tma_load_2d(k_s + half * (2 * kBlockN * 128), &tm_k, bars, half * 64, k_row);
-            tma_load_2d(k_s + half * (2 * kBlockN * 128) + kBlockN * 128, &tm_k, bars, half * 64, k_row + kBlockN);
-        }
-    } else if (warp == 1 && lane == 0) {
-        constexpr uint32_t idesc = make_idesc(kBlockM, 2 * kBlockN, false);
-        if (mbar_wait(bars, 0, abort_flag, status, 20)) {
-            tc_fence_after();
-#pragma unroll
-            for (int k = 0; k < D / 16; ++k) {
-                const uint32_t qa = smem_u32(q_s) + (k / 4) * (kBlockM * 128) + (k % 4) * 32;
-                const uint32_t ka = smem_u32(k_s) + (k / 4) * (2 * kBlockN * 128) + (k % 4) * 32;
-                mma_ss(tmem_base, smem_desc(qa, 0), smem_desc(ka, 0), idesc, k > 0 ? 1u : 0u);
+    if (warp == 0) {
+        if (lane == 0) {
+            int it = 0;
+            for (int n = blockIdx.x; n < n_tiles; n += gridDim.x, ++it) {
+                const int s = it & 1, ph = (it >> 1) & 1;
+                if (!mbar_wait(smem_free + s, ph ^ 1, abort_flag, status, 22)) break;
+                const int bh = n / n_row_blocks, R0 = (n - bh * n_row_blocks) * kBlockM;
+                const int b = bh / H, h = bh - b * H, kvh = h / (H / Hkv);
+                uint8_t *q_s = smem + s * P::kStage, *k_s = q_s + P::kQBytes;
+                mbar_expect_tx(full + s, P::kQBytes + P::kKBytes);
+                // rows before the start of K or of the previous head are masked by position in the epilogue
+                const int k_row = (b * Hkv + kvh) * N + R0 - kBlockN;
+                for (int half = 0; half < D / 64; ++half) {
+                    tma_load_2d(q_s + half * (kBlockM * 128), &tm_q, full + s, half * 64, bh * N + R0);
+                    // K-major operand of 256 rows: per 64-column half, rows 0..255 contiguous
+                    tma_load_2d(k_s + half * (2 * kBlockN * 128), &tm_k, full + s, half * 64, k_row);
+                    tma_load_2d(k_s + half * (2 * kBlockN * 128) + kBlockN * 128, &tm_k, full + s, half * 64, k_row + kBlockN);
+                }
             }
-            tc_commit(bars + 1);
+            // leave no copy in flight behind: every armed stage is waited for by the MMA warp in the normal
+            // course; after a failure wait (bounded) for the last one armed
+            if (*abort_flag && it > 0) mbar_wait_drain(full + ((it - 1) & 1), ((it - 1) >> 1) & 1);
         }
-    } else if (warp >= 2) {
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc(kBlockM, 2 * kBlockN, false);
+            int it = 0;
+            bool ok = true;
+            for (int n = blockIdx.x; n < n_tiles; n += gridDim.x, ++it) {
+                const int s = it & 1, ph = (it >> 1) & 1;
+                ok = mbar_wait(full + s, ph, abort_flag, status, 20) &&
+                     mbar_wait(tmem_free + s, ph ^ 1, abort_flag, status, 23);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t q_a = smem_u32(smem + s * P::kStage), k_a = q_a + P::kQBytes;
+#pragma unroll
+                for (int k = 0; k < D / 16; ++k) {
+                    const uint32_t qa = q_a + (k / 4) * (kBlockM * 128) + (k % 4) * 32;
+                    const uint32_t ka = k_a + (k / 4) * (2 * kBlockN * 128) + (k % 4) * 32;
+                    mma_ss(tmem_base + s * 256, smem_desc(qa, 0), smem_desc(ka, 0), idesc, k > 0 ? 1u : 0u);
+                }
+                tc_commit(mma_done + s);
+            }
+            // no MMA may still be running when tensor memory is freed: after a failure wait (bounded) for the
+            // last group issued (its commit covers everything before it)
+            if (!ok && it > 0) mbar_wait_drain(mma_done + ((it - 1) & 1), ((it - 1) >> 1) & 1);
+        }
+    } else {
+        const int g = (warp - 2) >> 2;                 // score group = stage = TMEM accumulator
         const int wq = warp & 3;                       // TMEM lane quarter this warp may read
-        const int r = wq * 32 + lane, t = R0 + r;
-        const uint32_t taddr = tmem_base + ((uint32_t)(wq * 32) << 16) + (uint32_t)(wq * 32 + kBlockN - C);
-        const bool ok = mbar_wait(bars + 1, 0, abort_flag, status, 21);
-        tc_fence_after();
-        float score = 0.f;
-        if (ok) {
-            // Element j of the warp's C+32 columns is the key at position R0 + 32 wq - C + j, and the window of
-            // the row in lane l is j in [l+1, l+C].  Columns [32, C) lie in every lane's window; of columns jj
-            // and C + jj (jj < 32) exactly one does (the first if jj > l).  So the first and the last block of
-            // 32 columns fold into one, and a row becomes C values without gaps: block 0 is the folded one (the
-            // token itself sits at jj = l), blocks 1 .. C/32-1 are columns [32 q, 32 q + 32).  Keys at negative
-            // positions (first tile of a sequence only) are set to -inf, which the exponential turns into 0.
-            constexpr int kBlocks = C / 32;
-            const bool first_tile = R0 == 0;
-            auto load_block = [&](int q, uint32_t (&v)[32]) {
-                tmem_ld32(taddr + q * 32, v);
-                if (q == 0) {
-                    uint32_t w[32];
-                    tmem_ld32(taddr + C, w);
-                    tmem_wait_ld();
+        const int r = wq * 32 + lane;                  // row of the tile owned by this thread
+        float *sc = reinterpret_cast<float *>(smem + P::kSc) + g * kBlockM;
+        uint32_t *ballots = reinterpret_cast<uint32_t *>(smem + P::kBallot) + g * 4;
+        const uint32_t taddr = tmem_base + g * 256 + ((uint32_t)(wq * 32) << 16) + (uint32_t)(wq * 32 + kBlockN - C);
+        const int group_bar = 1 + g;
+        int it = g, j = 0;
+        for (int n = blockIdx.x + g * gridDim.x; n < n_tiles; n += 2 * gridDim.x, it += 2, ++j) {
+            const int ph = j & 1;
+            const int bh = n / n_row_blocks, R0 = (n - bh * n_row_blocks) * kBlockM;
+            const int t = R0 + r;
+            bool ok = mbar_wait(mma_done + g, ph, abort_flag, status, 21);
+            // the group leaves the loop together
+            {
+                uint32_t all_ok;
+                asm volatile("{\n.reg .pred p, q;\nsetp.ne.b32 p, %1, 0;\nbarrier.cta.red.and.pred q, %2, 128, p;\nselp.b32 %0, 1, 0, q;\n}"
+                             : "=r"(all_ok) : "r"((uint32_t)ok), "r"(group_bar) : "memory");
+                ok = all_ok != 0;
+            }
+            if (!ok) break;
+            tc_fence_after();
+            if (r == 0) mbar_arrive(smem_free + g);    // the logits are complete: the stage's operands are free
+            float score = 0.f;
+            {
+                // Element j of the warp's C+32 columns is the key at position R0 + 32 wq - C + j, and the window of
+                // the row in lane l is j in [l+1, l+C].  Columns [32, C) lie in every lane's window; of columns jj
+                // and C + jj (jj < 32) exactly one does (the first if jj > l).  So the first and the last block of
+                // 32 columns fold into one, and a row becomes C values without gaps: block 0 is the folded one (the
+                // token itself sits at jj = l), blocks 1 .. C/32-1 are columns [32 q, 32 q + 32).  Keys at negative
+                // positions (first tile of a sequence only) are set to -inf, which the exponential turns into 0.
+                constexpr int kBlocks = C / 32;
+                const bool first_tile = R0 == 0;
+                auto load_block = [&](int q, uint32_t (&v)[32]) {
+                    tmem_ld32(taddr + q * 32, v);
+                    if (q == 0) {
+                        uint32_t w[32];
+                        tmem_ld32(taddr + C, w);
+                        tmem_wait_ld();
 #pragma unroll
-                    for (int jj = 0; jj < 32; ++jj) v[jj] = (jj > lane) ? v[jj] : w[jj];
+                        for (int jj = 0; jj < 32; ++jj) v[jj] = (jj > lane) ? v[jj] : w[jj];
+                    } else {
+                        tmem_wait_ld();
+                    }
+                    if (first_tile) {
+                        const int n_neg = C - wq * 32;   // columns below n_neg are before the start of the sequence
+#pragma unroll
+                        for (int jj = 0; jj < 32; ++jj)
+                            if (q * 32 + jj < n_neg && (q > 0 || jj > lane)) v[jj] = 0xff800000u;
+                    }
+                };
+                auto tmem_read_done = [&]() {   // the accumulator may be overwritten by the UMMA of the tile after next
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(tmem_free + g);
+                };
+                if constexpr (kBlocks == 2) {
+                    // the row fits the register file: one read of tensor memory, exponentials kept in place
+                    uint32_t v0[32], v1[32];
+                    load_block(0, v0);
+                    load_block(1, v1);
+                    tmem_read_done();
+                    float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+                    for (int jj = 0; jj < 32; jj += 2) {
+                        mx0 = max3(mx0, __uint_as_float(v0[jj]), __uint_as_float(v0[jj + 1]));
+                        mx1 = max3(mx1, __uint_as_float(v1[jj]), __uint_as_float(v1[jj + 1]));
+                    }
+                    const float neg_m = -fmaxf(mx0, mx1) * scale_log2;
+                    float z0 = 0.f, z1 = 0.f, e_self = 0.f;
+#pragma unroll
+                    for (int jj = 0; jj < 32; ++jj) {
+                        const float e0 = ex2(fmaf(__uint_as_float(v0[jj]), scale_log2, neg_m));
+                        const float e1 = ex2(fmaf(__uint_as_float(v1[jj]), scale_log2, neg_m));
+                        v1[jj] = __float_as_uint(e1);
+                        z1 += e1;
+                        if (jj == lane) e_self = e0;
+                        else z0 += e0;                    // the sum without the token itself is formed directly
+                        v0[jj] = __float_as_uint(e0);
+                    }
+                    const float z_nd = z0 + z1, z_all = z_nd + e_self;
+                    const float inv_all = 1.f / z_all, inv_nd = z_nd > 0.f ? 1.f / z_nd : 0.f;
+                    float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+                    for (int jj = 0; jj < 32; ++jj) {
+                        // a * ln((a + eps) / (b + eps)); a masked key has a = b = 0 and adds nothing
+                        const float e0 = __uint_as_float(v0[jj]), e1 = __uint_as_float(v1[jj]);
+                        const float a0 = e0 * inv_all, a1 = e1 * inv_all;
+                        const float b0 = (jj == lane) ? 0.f : e0 * inv_nd, b1 = e1 * inv_nd;
+                        s0 += a0 * (__log2f(a0 + eps) - __log2f(b0 + eps));
+                        s1 += a1 * (__log2f(a1 + eps) - __log2f(b1 + eps));
+                    }
+                    score = s0 + s1;
                 } else {
-                    tmem_wait_ld();
-                }
-                if (first_tile) {
-                    const int n_neg = C - wq * 32;   // columns below n_neg are before the start of the sequence
-#pragma unroll
-                    for (int jj = 0; jj < 32; ++jj)
-                        if (q * 32 + jj < n_neg && (q > 0 || jj > lane)) v[jj] = 0xff800000u;
-                }
-            };
-            if constexpr (kBlocks == 2) {
-                // the row fits the register file: one read of tensor memory, exponentials kept in place
-                uint32_t v0[32], v1[32];
-                load_block(0, v0);
-                load_block(1, v1);
-                float mx0 = -INFINITY, mx1 = -INFINITY;
-#pragma unroll
-                for (int jj = 0; jj < 32; jj += 2) {
-                    mx0 = max3(mx0, __uint_as_float(v0[jj]), __uint_as_float(v0[jj + 1]));
-                    mx1 = max3(mx1, __uint_as_float(v1[jj]), __uint_as_float(v1[jj + 1]));
-                }
-                const float neg_m = -fmaxf(mx0, mx1) * scale_log2;
-                float z0 = 0.f, z1 = 0.f, e_self = 0.f;
-#pragma unroll
-                for (int jj = 0; jj < 32; ++jj) {
-                    const float e0 = ex2(fmaf(__uint_as_float(v0[jj]), scale_log2, neg_m));
-                    const float e1 = ex2(fmaf(__uint_as_float(v1[jj]), scale_log2, neg_m));
-                    v1[jj] = __float_as_uint(e1);
-                    z1 += e1;
-                    if (jj == lane) e_self = e0;
-                    else z0 += e0;                    // the sum without the token itself is formed directly
-                    v0[jj] = __float_as_uint(e0);
-                }
-                const float z_nd = z0 + z1, z_all = z_nd + e_self;
-                const float inv_all = 1.f / z_all, inv_nd = z_nd > 0.f ? 1.f / z_nd : 0.f;
-                float s0 = 0.f, s1 = 0.f;
-#pragma unroll
-                for (int jj = 0; jj < 32; ++jj) {
-                    // a * ln((a + eps) / (b + eps)); a masked key has a = b = 0 and adds nothing
-                    const float e0 = __uint_as_float(v0[jj]), e1 = __uint_as_float(v1[jj]);
-                    const float a0 = e0 * inv_all, a1 = e1 * inv_all;
-                    const float b0 = (jj == lane) ? 0.f : e0 * inv_nd, b1 = e1 * inv_nd;
-                    s0 += a0 * (__log2f(a0 + eps) - __log2f(b0 + eps));
-                    s1 += a1 * (__log2f(a1 + eps) - __log2f(b1 + eps));
-                }
-                score = s0 + s1;
-            } else {
-                float mx = -INFINITY;
+                    float mx = -INFINITY;
 #pragma unroll 1
-                for (int q = 0; q < kBlocks; ++q) {
-                    uint32_t v[32];
-                    load_block(q, v);
+                    for (int q = 0; q < kBlocks; ++q) {
+                        uint32_t v[32];
+                        load_block(q, v);
 #pragma unroll
-                    for (int jj = 0; jj < 32; jj += 2) mx = max3(mx, __uint_as_float(v[jj]), __uint_as_float(v[jj + 1]));
-                }
-                const float neg_m = -mx * scale_log2;
-                float z_nd = 0.f, e_self = 0.f;
-#pragma unroll 1
-                for (int q = 0; q < kBlocks; ++q) {
-                    uint32_t v[32];
-                    load_block(q, v);
-#pragma unroll
-                    for (int jj = 0; jj < 32; ++jj) {
-                        const float e = ex2(fmaf(__uint_as_float(v[jj]), scale_log2, neg_m));
-                        if (q == 0 && jj == lane) e_self = e;
-                        else z_nd += e;
+                        for (int jj = 0; jj < 32; jj += 2) mx = max3(mx, __uint_as_float(v[jj]), __uint_as_float(v[jj + 1]));
                     }
-                }
-                const float z_all = z_nd + e_self;
-                const float inv_all = 1.f / z_all, inv_nd = z_nd > 0.f ? 1.f / z_nd : 0.f;
+                    const float neg_m = -mx * scale_log2;
+                    float z_nd = 0.f, e_self = 0.f;
 #pragma unroll 1
-                for (int q = 0; q < kBlocks; ++q) {
-                    uint32_t v[32];
-                    load_block(q, v);
+                    for (int q = 0; q < kBlocks; ++q) {
+                        uint32_t v[32];
+                        load_block(q, v);
 #pragma unroll
-                    for (int jj = 0; jj < 32; ++jj) {
-                        const float e = ex2(fmaf(__uint_as_float(v[jj]), scale_log2, neg_m));
-                        const float a = e * inv_all;
-                        const float bb = (q == 0 && jj == lane) ? 0.f : e * inv_nd;
-                        score += a * (__log2f(a + eps) - __log2f(bb + eps));
+                        for (int jj = 0; jj < 32; ++jj) {
+                            const float e = ex2(fmaf(__uint_as_float(v[jj]), scale_log2, neg_m));
+                            if (q == 0 && jj == lane) e_self = e;
+                            else z_nd += e;
+                        }
                     }
+                    const float z_all = z_nd + e_self;
+                    const float inv_all = 1.f / z_all, inv_nd = z_nd > 0.f ? 1.f / z_nd : 0.f;
+#pragma unroll 1
+                    for (int q = 0; q < kBlocks; ++q) {
+                        uint32_t v[32];
+                        load_block(q, v);
+#pragma unroll
+                        for (int jj = 0; jj < 32; ++jj) {
+                            const float e = ex2(fmaf(__uint_as_float(v[jj]), scale_log2, neg_m));
+                            const float a = e * inv_all;
+                            const float bb = (q == 0 && jj == lane) ? 0.f : e * inv_nd;
+                            score += a * (__log2f(a + eps) - __log2f(bb + eps));
+                        }
+                    }
+                    tmem_read_done();
+                }
+                score *= 0.6931471805599453f;
+            }
+            sc[r] = score;
+            if (t < N && scores != nullptr) scores[(long long)bh * N + t] = score;
+            asm volatile("bar.sync %0, 128;" ::"r"(group_bar) : "memory");
+            if (lam > 0) {
+                // top-k of each chunk of the tile: rank under (score descending, position ascending), NaN as -inf
+                const int cc = r / C, rr = r - cc * C;
+                const int n_c = min(C, N - (R0 + cc * C));   // tokens of this row's chunk (<= 0: past the end)
+                bool selected = false;
+                if (rr < n_c) {
+                    float mine = sc[r];
+                    if (isnan(mine)) mine = -INFINITY;
+                    int rank = 0;
+                    for (int jx = 0; jx < n_c; ++jx) {
+                        float o = sc[cc * C + jx];
+                        if (isnan(o)) o = -INFINITY;
+                        rank += (o > mine) || (o == mine && jx < rr);
+                    }
+                    selected = rank < lam;
+                }
+                // place of a selected row in the ascending output = selected rows before it in its chunk
+                const uint32_t votes = __ballot_sync(0xffffffffu, selected);
+                if (lane == 0) ballots[wq] = votes;
+                asm volatile("bar.sync %0, 128;" ::"r"(group_bar) : "memory");
+                if (n_c > 0) {
+                    int32_t *out = sel_idx + ((long long)bh * Tn + (R0 / C + cc)) * lam;
+                    int before = __popc(votes & ((1u << lane) - 1u));
+                    for (int w = cc * (C / 32); w < wq; ++w) before += __popc(ballots[w]);
+                    if (selected) out[before] = R0 + cc * C + rr;
+                    const int n_sel = n_c < lam ? n_c : lam;
+                    if (rr >= n_sel && rr < lam) out[rr] = -1;
                 }
             }
-            score *= 0.6931471805599453f;
+            // sc / ballots are written again in the group's next tile
+            asm volatile("bar.sync %0, 128;" ::"r"(group_bar) : "memory");
         }
-        sc[r] = score;
-        if (ok && t < N && scores != nullptr) scores[(long long)bh * N + t] = score;
     }
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, 256);
-    }
-    if (lam <= 0 || *abort_flag) return;
-    // top-k of each chunk of the tile: rank under (score descending, position ascending), NaN as -inf
-    const int tid = threadIdx.x;
-    int selected = 0, cc = 0, rr = 0, n_c = 0;
-    if (tid < kBlockM) {
-        cc = tid / C;
-        rr = tid - cc * C;
-        const int cbase = R0 + cc * C;
-        n_c = min(C, N - cbase);
-        if (rr < n_c) {
-            float mine = sc[tid];
-            if (isnan(mine)) mine = -INFINITY;
-            int rank = 0;
-            for (int j = 0; j < n_c; ++j) {
-                float o = sc[cc * C + j];
-                if (isnan(o)) o = -INFINITY;
-                rank += (o > mine) || (o == mine && j < rr);
-            }
-            selected = rank < lam;
-        }
-        flag[tid] = selected;
-    }
-    __syncthreads();
-    if (tid < kBlockM && n_c > 0) {
-        int32_t *out = sel_idx + ((long long)bh * Tn + (R0 / C + cc)) * lam;
-        int before = 0;
-        for (int j = 0; j < rr; ++j) before += flag[cc * C + j];
-        if (selected) out[before] = R0 + cc * C + rr;
-        const int n_sel = n_c < lam ? n_c : lam;
-        if (rr >= n_sel && rr < lam) out[rr] = -1;
+        tmem_dealloc(tmem_base, 512);
     }
 }
 
@@ -802,13 +871,20 @@ int launch_score_tc(const still_params_t *p, long long N, const void *Q, const v
     if (!make_map(&tq, Q, (unsigned long long)BH * N, D) ||
         !make_map(&tk, K, (unsigned long long)p->B * p->Hkv * N, D))
         return STILL_ERR_CUDA;
-    constexpr int kSmem = kBlockM * D * 2 + 2 * kBlockN * D * 2 + 16 + 16 + 2 * kBlockM * 4 + 1024;
+    constexpr int kSmem = ScoreSmem<D>::kAlloc;
     if (cudaFuncSetAttribute(score_select_tc_kernel<D, C>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) !=
         cudaSuccess)
         return STILL_ERR_CUDA;
-    dim3 grid((unsigned)((N + kBlockM - 1) / kBlockM), (unsigned)BH);
-    score_select_tc_kernel<D, C><<<grid, 192, kSmem, st>>>(tq, tk, scores, sel_idx, status, p->H, p->Hkv, (int)N,
-                                                           p->topk, p->sm_scale * 1.4426950408889634f, p->eps);
+    int dev = 0, n_sm = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n_sm <= 0)
+        return STILL_ERR_CUDA;
+    const long long n_row_blocks = (N + kBlockM - 1) / kBlockM, n_tiles = n_row_blocks * BH;
+    if (n_tiles >= (1ll << 31)) return STILL_ERR_UNSUPPORTED;
+    const unsigned grid = (unsigned)std::min<long long>(n_tiles, n_sm);   // one persistent CTA per SM
+    score_select_tc_kernel<D, C><<<grid, 320, kSmem, st>>>(tq, tk, scores, sel_idx, status, p->H, p->Hkv, (int)N,
+                                                           p->topk, p->sm_scale * 1.4426950408889634f, p->eps,
+                                                           (int)n_row_blocks, (int)n_tiles);
     ++*launches;
     return cudaGetLastError() == cudaSuccess ? STILL_OK : STILL_ERR_CUDA;
 }
