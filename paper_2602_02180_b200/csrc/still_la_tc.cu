@@ -261,6 +261,8 @@ struct ScanPlan {
     static constexpr int kMisc = kBar + kNumBars * 8;
     static constexpr int kTotal = kMisc + 16;
 };
+static_assert(ScanPlan<128>::kTotal <= 232448 && ScanPlan<256>::kTotal <= 232448,
+              "state scan: the shared-memory plan exceeds what a CTA can have");
 
 template <int NF>
 __global__ void __launch_bounds__(192, 1)

@@ -68,6 +68,14 @@ struct SmemPlan {
     static constexpr int kAlloc = kTotal + 1024;               // slack to align the base to 1024
 };
 
+constexpr int kMaxDynamicSmem = 232448;   // 227 KiB: the most a CTA can be given on sm_100
+static_assert(SmemPlan<64>::kAlloc <= kMaxDynamicSmem && SmemPlan<128>::kAlloc <= kMaxDynamicSmem,
+              "attention kernel: the shared-memory plan exceeds what a CTA can have");
+// every operand descriptor of the attention kernel addresses a whole tile inside its ring
+static_assert(SmemPlan<128>::kK == SmemPlan<128>::kQ + 2 * SmemPlan<128>::kTileBytes &&
+              SmemPlan<128>::kBar == SmemPlan<128>::kV + SmemPlan<128>::kVStages * SmemPlan<128>::kTileBytes,
+              "attention kernel: rings must follow each other without gaps");
+
 // Per-CTA description of the key stream.
 struct Stream {
     int n_sel_a, n_sel_b;   // SEL tiles used by tile A / tile B
@@ -533,6 +541,9 @@ struct ScoreSmem {
     static constexpr int kTotal = kBallot + 2 * 4 * 4;
     static constexpr int kAlloc = kTotal + 1024;     // slack to align the base to 1024
 };
+
+static_assert(ScoreSmem<64>::kAlloc <= kMaxDynamicSmem && ScoreSmem<128>::kAlloc <= kMaxDynamicSmem,
+              "score kernel: two stages must fit one CTA's shared memory");
 
 template <int D, int C>
 __global__ void __launch_bounds__(320, 1)
