@@ -12,9 +12,9 @@ from tests import util_parity as U
 pytestmark = pytest.mark.gpu
 
 
-def _decode_case(w, n0, n_steps, gate=False, tweak=None):
-    """Prefill n0 tokens into a state, decode n_steps more, compare every decoded row with
-    the oracle's chunk-wise form over the whole sequence (the GPU's selection forced)."""
+def _decode_case(w, n0, n_steps, gate=False, tweak=None, expect_ties=False, n_heads=4, want_y=True):
+    """Prefill n0 tokens into a state, decode n_steps more, compare every decoded row of the sampled heads
+    with the oracle's chunk-wise form over the whole sequence (the GPU's selection forced)."""
     dev = "cuda"
     N = n0 + n_steps
     wN = w.with_(N=N)
@@ -23,14 +23,22 @@ def _decode_case(w, n0, n_steps, gate=False, tweak=None):
         Q, K, V = tweak(Q, K, V)
     Wq, Wk = synth.make_npmap_weights(wN, dev)
     G = synth.make_gate(wN, dev) if gate else None
+    rep = w.H // w.Hkv
+    heads = U.sample_heads(w, n_heads)
+    # what the oracle needs of the sampled heads, and the decode steps' inputs; the whole-sequence device
+    # tensors go before the prefill allocates its workspace (the full-size case would not fit otherwise)
+    host = {(b, h): (U.f64(Q[b, h]), U.f64(K[b, h // rep]), U.f64(V[b, h // rep]),
+                     None if G is None else U.f64(G[b, h])) for b, h in heads}
+    step_in = [t[:, :, n0:].permute(2, 0, 1, 3).contiguous() if t is not None else None for t in (Q, K, V, G)]  # [steps,B,heads,d]
+    pre = [t[:, :, :n0].contiguous() if t is not None else None for t in (Q, K, V, G)]
+    del Q, K, V, G
     p = U.params_of(w)
     cap = N + 5
     lay = still.state_layout(p, cap)
     state = torch.zeros(lay["total"], dtype=torch.uint8, device=dev)
     if n0 > 0:
-        still.hybrid_attn_fwd(p, Q[:, :, :n0].contiguous(), K[:, :, :n0].contiguous(), V[:, :, :n0].contiguous(),
-                              Wq, Wk, G=None if G is None else G[:, :, :n0].contiguous(), state=state,
-                              state_max_tokens=cap)
+        still.hybrid_attn_fwd(p, pre[0], pre[1], pre[2], Wq, Wk, G=pre[3], state=state, state_max_tokens=cap,
+                              want_y=want_y)
     else:
         # an empty prefill initialises the state
         c = p.c()
@@ -39,11 +47,13 @@ def _decode_case(w, n0, n_steps, gate=False, tweak=None):
             ctypes.byref(c), 0, None, None, None, None, None, None, None, None, None, None, None,
             ctypes.c_void_p(state.data_ptr()), cap, None, 0, None)
         assert rc == 0
+    torch.cuda.synchronize()
+    del pre
+    torch.cuda.empty_cache()
     ys = []
-    for t in range(n0, N):
-        y = still.hybrid_attn_step(p, state, cap, t, Q[:, :, t].contiguous(), K[:, :, t].contiguous(),
-                                   V[:, :, t].contiguous(), Wq, Wk,
-                                   g=None if G is None else G[:, :, t].contiguous())
+    for i in range(n_steps):
+        y = still.hybrid_attn_step(p, state, cap, n0 + i, step_in[0][i], step_in[1][i], step_in[2][i], Wq, Wk,
+                                   g=None if step_in[3] is None else step_in[3][i])
         ys.append(y)
     torch.cuda.synchronize()
     assert still.device_status(state) == (0, 0)
@@ -55,13 +65,17 @@ def _decode_case(w, n0, n_steps, gate=False, tweak=None):
     sel = None
     if lam > 0:
         sel = state[lay["sel_idx"]: lay["sel_idx"] + w.B * w.H * capT * lam * 4].view(torch.int32).view(w.B, w.H, capT, lam)
-    rep = w.H // w.Hkv
     rows = list(range(n0, N))
     hp = oracle.HeadParams(C, lam, w.sm_scale)
-    T = -(-N // C)
-    for b, h in U.sample_heads(w, 4):
+    tie_seen = False
+    worst = 0.0
+    for b, h in heads:
         kv = h // rep
+        q64, k64, v64, g64 = host[(b, h)]
         scores = sc[b, h, :N].cpu().numpy().astype(np.float64)
+        if expect_ties and n_routed > 0:
+            ch = np.sort(scores[: n_routed * C].reshape(n_routed, C)[n0 // C:], axis=1)   # chunks routed by decode steps
+            tie_seen |= bool(np.any(np.diff(ch, axis=1) == 0))
         forced = None
         if lam > 0:
             want = oracle.select(scores, C, lam)
@@ -69,11 +83,14 @@ def _decode_case(w, n0, n_steps, gate=False, tweak=None):
             np.testing.assert_array_equal(got, want[:n_routed])  # bit-exact on the GPU's own scores
             forced = want.copy()
             forced[:n_routed] = got
-        out = oracle.chunkwise(U.f64(Q[b, h]), U.f64(K[b, kv]), U.f64(V[b, kv]), U.f64(Wq[h]), U.f64(Wk[kv]), hp,
-                               g=None if G is None else U.f64(G[b, h]), forced_idx=forced, rows=rows)
-        assert np.abs(scores - out["score"]).max() < (1e-4 if w.dtype == "fp32" else 1e-3)
+        out = oracle.chunkwise(q64, k64, v64, U.f64(Wq[h]), U.f64(Wk[kv]), hp, g=g64, forced_idx=forced, rows=rows)
+        serr = np.abs(scores - out["score"]).max()
+        assert serr <= U.SCORE_TOL[w.torch_dtype], f"b={b} h={h} score max-abs {serr:.3e}"
         err = np.abs(U.f64(Yd[b, h]) - out["y"]).max()
+        worst = max(worst, err)
         assert err <= U.TOL[w.torch_dtype], f"b={b} h={h} max-abs {err:.3e}"
+    assert tie_seen or not expect_ties, "the constructed input produced no tie in a chunk routed by a decode step"
+    return worst
 
 
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
@@ -111,11 +128,30 @@ def test_decode_with_growing_logits(k):
     _decode_case(w, 128 * 5 + 9, 70, tweak=tweak)
 
 
-def test_c5_full_size_sampled():
+@pytest.mark.parametrize("dtype,C,k", [("bf16", 64, 16), ("bf16", 32, 8), ("fp32", 32, 8)])
+@pytest.mark.parametrize("case", ["zero_queries", "periodic_tokens"])
+def test_decode_routing_breaks_ties_like_the_oracle(dtype, C, k, case):
+    # Equal scores inside a chunk (all logits zero, or tokens repeating with period 16): the chunk routed at a
+    # decode step must be ranked under (score descending, position ascending), as the prefill does.
+    def tweak(Q, K, V):
+        if case == "zero_queries":
+            return torch.zeros_like(Q), K, V
+        reps = -(-Q.shape[2] // 16)
+        rep = lambda x: x[:, :, :16].repeat(1, 1, reps, 1)[:, :, : x.shape[2]].contiguous()  # noqa: E731
+        return rep(Q), rep(K), V
+
+    w = synth.Workload("t", 1, 4, 2, 64, 0, C, k, dtype, "iid", 31)
+    _decode_case(w, C + 7, 4 * C + 3, tweak=tweak, expect_ties=True)
+
+
+@pytest.mark.parametrize("k,steps", [(64, 256), (16, 136)])
+def test_c5_full_size_sampled(k, steps):
     # The decode workload as benchmarked: batch 64, 32768-token prefix summarised by the prefill into the
-    # decode state, then a few steps; sampled (batch, head) pairs against the oracle.
-    w = synth.WORKLOADS["c5"]
-    _decode_case(w, w.N, 3)
+    # decode state, then the benchmark's 256 steps (four chunks are routed on the way) with every token
+    # selected, and 136 steps (two routings) of the lambda = C/4 companion; sampled (batch, head) pairs
+    # against the oracle.
+    w = synth.WORKLOADS["c5"].with_(k=k)
+    _decode_case(w, w.N, steps, n_heads=4 if k == 64 else 3, want_y=False)
 
 
 def test_state_full_and_mismatch():

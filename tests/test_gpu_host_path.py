@@ -9,10 +9,13 @@ from tests import util_parity as U
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("B,H,Hkv,N,k", [(2, 8, 4, 64 * 6, 16), (1, 4, 2, 64 * 5 + 3, 16), (3, 4, 4, 256, 64)])
-def test_host_buffers_match_device_buffers(B, H, Hkv, N, k):
-    # pipelined over (batch, KV-head group) parts when the slices are aligned, single shot otherwise
-    w = synth.Workload("h", B, H, Hkv, 64, N, 64, k, "bf16", "iid", 77)
+@pytest.mark.parametrize("B,H,Hkv,d,N,k", [(2, 8, 4, 64, 64 * 6, 16), (1, 4, 2, 64, 64 * 5 + 3, 16), (3, 4, 4, 64, 256, 64),
+                                           (2, 32, 8, 128, 64 * 20, 64), (2, 32, 8, 128, 64 * 12, 16)])
+def test_host_buffers_match_device_buffers(B, H, Hkv, d, N, k):
+    # pipelined over (batch, KV-head group) parts when the slices are aligned, single shot otherwise; the
+    # last two cases have the benchmark's head structure (batch 2 x 8 KV heads x 4 query heads, d = 128:
+    # sixteen parts computing alternately on two streams with a workspace each)
+    w = synth.Workload("h", B, H, Hkv, d, N, 64, k, "bf16", "iid", 77)
     Q, K, V = synth.make_qkv(w, "cuda")
     Wq, Wk = synth.make_npmap_weights(w, "cuda")
     G = synth.make_gate(w, "cuda")

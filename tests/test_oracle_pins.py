@@ -190,6 +190,18 @@ def test_npmap_u_norm_equals_input_norm():
     np.testing.assert_allclose(u_norm, np.linalg.norm(x, axis=1), rtol=1e-10)
 
 
+def test_npmap_zero_map_gives_uniform_features():
+    # f(x) = 0 (W = 0, no bias): the direction of f is undefined; the norm in the denominator is
+    # clamped, so u = 0 and both softmaxes are uniform, 1 / d_f each -- whatever the norm of x.
+    d, df = 6, 5
+    x = RNG.standard_normal((7, d)) * np.array([1e-3, 1.0, 50.0, 1.0, 1.0, 1e3, 1.0])[:, None]
+    phi = o.npmap(x, np.zeros((d, df)))
+    np.testing.assert_allclose(phi, 1.0 / df, rtol=0, atol=1e-15)
+    # a zero input row with any map: f = 0 and ||x|| = 0, again uniform
+    phi0 = o.npmap(np.zeros((2, d)), RNG.standard_normal((d, df)))
+    np.testing.assert_allclose(phi0, 1.0 / df, rtol=0, atol=1e-15)
+
+
 # --------------------------------------------------------------------------- whole layer
 
 
@@ -431,3 +443,27 @@ def test_layer_gqa_mapping():
             one = o.chunkwise(Q[b, h], K[b, h // 2], V[b, h // 2], Wq[h], Wk[h // 2], p)
             np.testing.assert_array_equal(out["y"][b, h], one["y"])
             np.testing.assert_array_equal(out["idx"][b, h], one["idx"])
+
+
+def test_layer_forced_indices_are_taken_per_head():
+    # forced_idx [B,H,T,lam]: head (b,h) must use its own slice (a wrong offset would show as another
+    # head's selection, or as the head's own top-lambda)
+    B, H, Hkv, N, d, C, lam = 2, 2, 1, 48, 4, 8, 2
+    Q = RNG.standard_normal((B, H, N, d))
+    K, V = RNG.standard_normal((2, B, Hkv, N, d))
+    Wq = RNG.standard_normal((H, d, d))
+    Wk = RNG.standard_normal((Hkv, d, d))
+    p = o.HeadParams(C, lam, 0.5)
+    T = N // C
+    forced = np.empty((B, H, T, lam), dtype=np.int32)
+    for b in range(B):
+        for h in range(H):
+            for c in range(T):
+                forced[b, h, c] = c * C + np.array([(b + 2 * h) % C, (b + 2 * h + 3) % C])
+    forced.sort(axis=-1)
+    out = o.layer(Q, K, V, Wq, Wk, p, forced_idx=forced)
+    for b in range(B):
+        for h in range(H):
+            one = o.chunkwise(Q[b, h], K[b, 0], V[b, 0], Wq[h], Wk[0], p, forced_idx=forced[b, h])
+            np.testing.assert_array_equal(out["y"][b, h], one["y"])
+            np.testing.assert_array_equal(out["idx"][b, h], forced[b, h])

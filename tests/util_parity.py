@@ -10,6 +10,9 @@ from oracle import still_oracle as oracle
 from paper_2602_02180_b200 import synth
 
 TOL = {torch.float32: 1e-4, torch.bfloat16: 2e-2}  # max-abs on Y, per dtype
+# max-abs on the Self-Saliency Score against the oracle's (same rounded inputs on both sides; the kernels
+# use the hardware's approximate exp2 / log2, and scores reach log((1 + eps) / eps) = 13.8)
+SCORE_TOL = {torch.float32: 1e-4, torch.bfloat16: 2e-3}
 
 
 def f64(t):
@@ -29,10 +32,24 @@ def check_selection(scores, sel_idx, C, lam, heads):
         np.testing.assert_array_equal(si[b, h], want, err_msg=f"selection differs at b={b} h={h}")
 
 
+def jaccard(a, b):
+    """Mean Jaccard index over chunks of two [T, lam] selections (-1 = padding)."""
+    vals = []
+    for ra, rb in zip(np.asarray(a), np.asarray(b)):
+        sa, sb = set(ra[ra >= 0].tolist()), set(rb[rb >= 0].tolist())
+        if sa or sb:
+            vals.append(len(sa & sb) / len(sa | sb))
+    return float(np.mean(vals)) if vals else 1.0
+
+
 def check_outputs(w, Q, K, V, Wq, Wk, Y, scores, sel_idx, heads, rows=None, G=None, bq=None, bk=None,
-                  tol=None, eps=1e-6):
-    """Y of the sampled heads (and rows) against the oracle run with the GPU's selection."""
+                  tol=None, eps=1e-6, score_tol=None, report=None):
+    """Y of the sampled heads (and rows) against the oracle run with the GPU's selection, and the GPU's
+    scores against the oracle's.  Returns (worst Y error, worst score error); `report`, if a dict, also
+    receives the Jaccard agreement between the oracle's own selection and the GPU's (reported, not gated:
+    near-ties may flip)."""
     tol = TOL[w.torch_dtype] if tol is None else tol
+    score_tol = SCORE_TOL[w.torch_dtype] if score_tol is None else score_tol
     rep = w.H // w.Hkv
     p = oracle.HeadParams(w.C, w.k, w.sm_scale, eps)
     worst = 0.0
@@ -49,8 +66,13 @@ def check_outputs(w, Q, K, V, Wq, Wk, Y, scores, sel_idx, heads, rows=None, G=No
         assert np.all(np.isfinite(got)), f"non-finite output at b={b} h={h}"
         err = np.abs(got - out["y"]).max()
         worst = max(worst, err)
-        score_err = max(score_err, np.abs(scores[b, h].cpu().numpy() - out["score"]).max())
+        serr = np.abs(scores[b, h].cpu().numpy() - out["score"]).max()
+        score_err = max(score_err, serr)
         assert err <= tol, f"b={b} h={h}: max-abs {err:.3e} > {tol}"
+        assert serr <= score_tol, f"b={b} h={h}: score max-abs {serr:.3e} > {score_tol}"
+        if report is not None and w.k > 0:
+            pure = oracle.select(out["score"], w.C, w.k)
+            report.setdefault("jaccard", []).append(jaccard(pure, sel_idx[b, h].cpu().numpy()))
     return worst, score_err
 
 
