@@ -23,7 +23,15 @@
  * General conventions
  *   - Every tensor pointer is DEVICE memory owned by the caller, contiguous in
  *     the stated layout, aligned to 16 bytes.  The library allocates no device
- *     memory and keeps no global state.
+ *     memory.  What it keeps between calls is host-side and per host thread:
+ *     encoded TMA descriptors of recently used buffers, the launch count and
+ *     the timing events of still_profile_*, and -- only after a call of
+ *     still_hybrid_attn_fwd_host -- three side streams and the events that
+ *     order them, created on first use and kept until the thread exits.
+ *     still_hybrid_attn_fwd_static adds one fixed array in the library's device
+ *     image (see there).
+ *   - The device that is current when a call is made must be the device of
+ *     `cuda_stream` and of every buffer.
  *   - Calls enqueue work on `cuda_stream` (a cudaStream_t passed as void*, NULL =
  *     the legacy default stream) and return without synchronising.
  *   - Return value: STILL_OK (0) or a negative still_status code.  No C++
@@ -62,9 +70,12 @@ enum { STILL_DTYPE_FP32 = 0, STILL_DTYPE_BF16 = 1 };
  * phi_q / phi_k, chunk size C, number lambda, small constant epsilon).
  *
  * Supported: d in {64, 128}; d_f in {32, 64, 128} with d_f <= d; chunk in
- * {64, 128}; 0 <= topk <= chunk; dtype fp32 or bf16.  bf16 inputs run on the
- * tcgen05 tensor-core kernels, fp32 inputs on fp32 FMA kernels (TF32 would not
- * meet the 1e-4 output tolerance).
+ * {32, 64, 128}; 0 <= topk <= chunk; dtype fp32 or bf16.  bf16 inputs with
+ * chunk 64 or 128 run on the tcgen05 tensor-core kernels (the linear branch
+ * too when d_f >= 64); fp32 inputs, and bf16 inputs with chunk 32, run on fp32
+ * FMA kernels (TF32 would not meet the 1e-4 output tolerance of fp32).  The
+ * bf16 decode step packs the query heads of a KV head into one tensor-core
+ * tile and needs H / Hkv <= 16.
  */
 typedef struct still_params {
     int32_t B;          /* batch                                                             */
@@ -141,7 +152,10 @@ int still_state_layout(const still_params_t *p, int64_t max_tokens, still_state_
  *   workspace, workspace_bytes  at least still_workspace_bytes(p, N)
  *
  * Ties in the score are broken by position (smaller first); NaN scores rank
- * lowest.  N need not be a multiple of chunk.  N = 0 is a no-op.
+ * lowest.  N need not be a multiple of chunk.  N = 0 launches nothing, except
+ * that with state_out it initialises the state to "no tokens" (header, zero S
+ * and z), which is how a decode from an empty sequence starts; the tensor
+ * pointers may then be NULL.
  * Errors: STILL_ERR_INVALID_ARG, STILL_ERR_UNSUPPORTED,
  * STILL_ERR_WORKSPACE_TOO_SMALL, STILL_ERR_STATE_FULL (N > capacity),
  * STILL_ERR_CUDA.
@@ -155,8 +169,14 @@ int still_hybrid_attn_fwd(const still_params_t *p, int64_t N, const void *Q, con
 /*
  * Decode: one step of the Recurrent Form (Sec. 3.3) for every sequence of the
  * batch.  t_pos is the number of tokens the state already holds (the new token
- * gets 0-based position t_pos); the caller tracks it on the host and it must
- * match the state (a mismatch is recorded in the state's status word).
+ * gets 0-based position t_pos); the caller tracks it on the host.  The first
+ * kernel of the step compares the state's header with the call -- magic word,
+ * the parameters and capacity the state was built with, the token count -- and
+ * on a mismatch the step writes nothing (state and y unchanged) and records
+ * STILL_ERR_STATE_MISMATCH in the state's status word (detail 1: token count,
+ * 2: not a state, 3: other parameters); still_device_status reads it.  Once
+ * the status word is set every later step on that state is a no-op, until a
+ * prefill rebuilds the state.
  *
  *   q [B, H, d], k, v [B, Hkv, d], g [B, H, d] or NULL, y [B, H, d]
  *   Wq, bq, Wk, bk as for the prefill
@@ -207,8 +227,8 @@ int still_hybrid_attn_fwd_host(const still_params_t *p, int64_t N, const void *h
  *   - Arguments are those of still_hybrid_attn_fwd without state_out, workspace and their sizes;
  *     Q, K, V, (G, Wq, bq, Wk, bk), Y, scores, sel_idx are still the caller's device buffers.
  *   - Limit: still_workspace_bytes(p, N) must not exceed STILL_STATIC_WORKSPACE_BYTES, otherwise
- *     the call returns STILL_ERR_WORKSPACE_TOO_SMALL and launches nothing.  (With the default
- *     d_f = d = 64, bf16, B = 1, H = 4 and topk = chunk / 4 this admits N up to about 5000.)
+ *     the call returns STILL_ERR_WORKSPACE_TOO_SMALL and launches nothing.  still_workspace_bytes
+ *     tells in advance (it is host arithmetic); the workspace grows with B * H * N.
  *   - The first call on each device looks up the array's device address (one
  *     cudaGetSymbolAddress, with that device current); make that first call outside any stream
  *     capture.
@@ -237,6 +257,16 @@ int still_device_status(const void *workspace_or_state, void *cuda_stream, int *
 /* Number of kernel launches the last still_hybrid_attn_fwd / _step call on this
  * host thread enqueued (for launch accounting in benchmarks). */
 int still_last_launch_count(void);
+
+/*
+ * Self-test of the bounded device-side wait.  Launches one small kernel whose only act is the
+ * mbarrier wait of the tensor-core kernels on a barrier that nothing ever arrives on, with a limit
+ * of `limit_cycles` SM clock cycles instead of the kernels' built-in limit.  The wait runs out, the
+ * kernel records STILL_ERR_DEVICE_TIMEOUT with detail 99 in `status_block` (256 bytes of device
+ * memory, 16-byte aligned, cleared by this call) and ends normally; still_device_status(status_block)
+ * then reports it.  The context stays usable.  Errors: STILL_ERR_INVALID_ARG, STILL_ERR_CUDA.
+ */
+int still_selftest_wait_timeout(void *status_block, int64_t limit_cycles, void *cuda_stream);
 
 /*
  * Optional timing of the dominant kernel (the softmax-attention + merge kernel of the

@@ -11,6 +11,7 @@ from .binding import (  # noqa: F401
     last_launch_count,
     profile_collect,
     profile_enable,
+    selftest_wait_timeout,
     state_bytes,
     state_layout,
     strerror,

@@ -96,6 +96,8 @@ def lib():
         L.still_device_status.restype = ctypes.c_int
         L.still_device_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_int)]
         L.still_last_launch_count.restype = ctypes.c_int
+        L.still_selftest_wait_timeout.restype = ctypes.c_int
+        L.still_selftest_wait_timeout.argtypes = [vp, i64, vp]
         L.still_profile_enable.restype = ctypes.c_int
         L.still_profile_enable.argtypes = [ctypes.c_int]
         L.still_profile_collect.restype = ctypes.c_int
@@ -246,6 +248,13 @@ def profile_collect(capacity: int = 4096) -> list[float]:
     if rc != STILL_OK:
         raise StillError(rc, "still_profile_collect")
     return [buf[i] for i in range(n.value)]
+
+
+def selftest_wait_timeout(status_block, limit_cycles: int) -> None:
+    """still_selftest_wait_timeout: a bounded device wait that runs out after limit_cycles."""
+    rc = lib().still_selftest_wait_timeout(_ptr(status_block), int(limit_cycles), _stream())
+    if rc != STILL_OK:
+        raise StillError(rc, "still_selftest_wait_timeout")
 
 
 def device_status(buf) -> tuple[int, int]:

@@ -28,8 +28,7 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
     if force or _stale():
         nvcc = os.environ.get("NVCC", "nvcc")
         tmp = LIB_PATH + f".{os.getpid()}.tmp"
-        extra = os.environ.get("STILL_NVCC_EXTRA", "").split()  # e.g. -DSTILL_EXP2_POLY_PAIRS=2
-        cmd = [nvcc] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp]
+        cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp]
         cmd += [os.path.join(CSRC, s) for s in SOURCES]
         subprocess.check_call(cmd)
         os.replace(tmp, LIB_PATH)

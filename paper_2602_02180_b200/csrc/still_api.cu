@@ -276,7 +276,6 @@ static int fwd_typed(const still_params_t *p, long long N, const T *Q, const T *
     float *S_out = state ? reinterpret_cast<float *>(state + L.S) : nullptr;
     float *z_out = state ? reinterpret_cast<float *>(state + L.z) : nullptr;
     if (w.la) {
-        if (!Wq || !Wk) return STILL_ERR_INVALID_ARG;
         T *phiQ = reinterpret_cast<T *>(ws + w.phiQ), *phiK = reinterpret_cast<T *>(ws + w.phiK);
         nla = reinterpret_cast<float *>(ws + w.nla);
         dla = reinterpret_cast<float *>(ws + w.dla);
@@ -396,6 +395,12 @@ int still_hybrid_attn_fwd(const still_params_t *p, int64_t N, const void *Q, con
         if (ptr && misaligned(ptr)) return STILL_ERR_INVALID_ARG;
     FwdPlan w = plan_fwd(p, N);
     if (workspace_bytes < w.total) return STILL_ERR_WORKSPACE_TOO_SMALL;
+    if (w.la && (!Wq || !Wk)) return STILL_ERR_INVALID_ARG;   // the linear branch needs both maps
+    if (state_out) {
+        still_state_layout_t L{};
+        if ((rc = plan_state(p, state_max_tokens, &L)) != STILL_OK) return rc;
+        if (N > L.capacity) return STILL_ERR_STATE_FULL;
+    }
     cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
     char *ws = reinterpret_cast<char *>(workspace);
     char *state = reinterpret_cast<char *>(state_out);
@@ -516,18 +521,19 @@ int still_hybrid_attn_fwd_host(const still_params_t *p, int64_t N, const void *h
         STILL_CUDA(cudaStreamSynchronize(st));
         return STILL_OK;
     }
-    cudaEvent_t ev_start, ev_in[kMaxParts], ev_done[kMaxParts];
-    STILL_CUDA(cudaEventCreateWithFlags(&ev_start, cudaEventDisableTiming));
+    // Events of the pipeline: created on first use per host thread and kept, like the side streams.
+    static thread_local cudaEvent_t ev_start = nullptr, ev_in[kMaxParts] = {}, ev_done[kMaxParts] = {};
+    if (!ev_start) STILL_CUDA(cudaEventCreateWithFlags(&ev_start, cudaEventDisableTiming));
     for (int i = 0; i < n_parts; ++i) {
-        STILL_CUDA(cudaEventCreateWithFlags(&ev_in[i], cudaEventDisableTiming));
-        STILL_CUDA(cudaEventCreateWithFlags(&ev_done[i], cudaEventDisableTiming));
+        if (!ev_in[i]) STILL_CUDA(cudaEventCreateWithFlags(&ev_in[i], cudaEventDisableTiming));
+        if (!ev_done[i]) STILL_CUDA(cudaEventCreateWithFlags(&ev_done[i], cudaEventDisableTiming));
     }
+    // after a failure, whatever was enqueued drains before the call returns (the host buffers are the caller's)
     auto cleanup = [&]() {
-        cudaEventDestroy(ev_start);
-        for (int i = 0; i < n_parts; ++i) {
-            cudaEventDestroy(ev_in[i]);
-            cudaEventDestroy(ev_done[i]);
-        }
+        cudaStreamSynchronize(s_in);
+        cudaStreamSynchronize(st);
+        cudaStreamSynchronize(s_alt);
+        cudaStreamSynchronize(s_out);
     };
     // the side streams start after what the caller has already enqueued (and after the weights)
     STILL_CUDA(cudaEventRecord(ev_start, st));
@@ -577,10 +583,9 @@ int still_hybrid_attn_fwd_host(const still_params_t *p, int64_t N, const void *h
             e = cudaMemcpyAsync(reinterpret_cast<char *>(hsel_idx) + i * si_part, dsi + i * si_part, si_part, cudaMemcpyDeviceToHost, s_out);
         if (e != cudaSuccess) rc = STILL_ERR_CUDA;
     }
-    // everything enqueued has to drain before the events go and before the host reads the outputs
+    // everything enqueued has to drain before the host reads the outputs
     cudaError_t e1 = cudaStreamSynchronize(s_in), e2 = cudaStreamSynchronize(st), e3 = cudaStreamSynchronize(s_alt);
     cudaError_t e4 = cudaStreamSynchronize(s_out);
-    cleanup();
     if (rc != STILL_OK) return rc;
     if (e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess || e4 != cudaSuccess) return STILL_ERR_CUDA;
     return STILL_OK;
@@ -600,6 +605,13 @@ int still_device_status(const void *workspace_or_state, void *cuda_stream, int *
 }
 
 int still_last_launch_count(void) { return g_launches; }
+
+int still_selftest_wait_timeout(void *status_block, int64_t limit_cycles, void *cuda_stream) {
+    if (!status_block || misaligned(status_block) || limit_cycles <= 0) return STILL_ERR_INVALID_ARG;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    STILL_CUDA(cudaMemsetAsync(status_block, 0, 256, st));
+    return tc_selftest_wait_timeout(reinterpret_cast<int *>(status_block), limit_cycles, st);
+}
 
 int still_profile_enable(int max_records) {
     if (max_records <= 0 || g_prof_ev) return STILL_ERR_INVALID_ARG;

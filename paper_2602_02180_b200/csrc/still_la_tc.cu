@@ -559,7 +559,7 @@ int launch_npmap(const void *X, const void *W, const void *bias, void *phi, int 
         !make_map_2d(&tw, W, (unsigned long long)heads * D, DF, D, false))
         return STILL_ERR_CUDA;
     constexpr int kSmem = NpmapSmem<D, DF, TOut>::kTotal;
-    if (cudaFuncSetAttribute(npmap_tc_kernel<D, DF, TOut>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) !=
+    if (ensure_dynamic_smem((const void *)npmap_tc_kernel<D, DF, TOut>, kSmem) !=
         cudaSuccess)
         return STILL_ERR_CUDA;
     dim3 grid((unsigned)((N + 127) / 128), (unsigned)heads, (unsigned)B);
@@ -587,7 +587,7 @@ int launch_scan(const still_params_t *p, long long N, const void *phiQ, const vo
     if (!make_map_2d(&tk, phiK, BHkv * N, NF, 64, false) || !make_map_2d(&tv, V, BHkv * N, p->d, 64, false) ||
         !make_map_2d(&tq, phiQ, BH * N, NF, 64, true))
         return STILL_ERR_CUDA;
-    if (cudaFuncSetAttribute(la_scan_tc_kernel<NF>, cudaFuncAttributeMaxDynamicSharedMemorySize, ScanPlan<NF>::kTotal) !=
+    if (ensure_dynamic_smem((const void *)la_scan_tc_kernel<NF>, ScanPlan<NF>::kTotal) !=
         cudaSuccess)
         return STILL_ERR_CUDA;
     dim3 grid((unsigned)BH, (unsigned)(p->d / 64));

@@ -48,9 +48,9 @@ extern "C" int still_hybrid_attn_fwd_static(const still_params_t *p, int64_t N, 
                                             const void *Wk, const void *bk, void *Y, float *scores,
                                             int32_t *sel_idx, void *cuda_stream) {
     if (!p || N < 0) return STILL_ERR_INVALID_ARG;
-    if (N == 0) return STILL_OK;
     const size_t need = still_workspace_bytes(p, N);
     if (need == 0) return STILL_ERR_INVALID_ARG;  // parameters the prefill would reject as well
+    if (N == 0) return STILL_OK;
     if (need > (size_t)STILL_STATIC_WORKSPACE_BYTES) return STILL_ERR_WORKSPACE_TOO_SMALL;
     void *ws = static_workspace_ptr();
     if (!ws) return STILL_ERR_CUDA;

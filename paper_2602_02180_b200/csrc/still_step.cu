@@ -51,18 +51,44 @@ __device__ __forceinline__ void load_vec<4, __nv_bfloat16>(const __nv_bfloat16 *
     out[0] = a.x; out[1] = a.y; out[2] = b.x; out[3] = b.y;
 }
 
-// grid (H, B), 32 threads: one warp scores the new token of one query head.
+// What a step expects to find in the header of the decode state.
+struct StateKey {
+    int32_t B, H, Hkv, d, d_f, chunk, topk, dtype;
+    long long cap, t;
+};
+
+// Header words 0-13 against the call: 0 if they agree, else a detail code (1: token count, 2: not a
+// state / other layout version, 3: built with other parameters or another capacity, 4: an earlier step
+// has already failed).  Nothing writes these words while the first kernel of a step runs.
+__device__ __forceinline__ int state_mismatch(const int32_t *hdr, const StateKey &k) {
+    if (hdr[0] != 0x5354494c || hdr[1] != 1) return 2;
+    if (hdr[2] != k.B || hdr[3] != k.H || hdr[4] != k.Hkv || hdr[5] != k.d || hdr[6] != k.d_f || hdr[7] != k.chunk ||
+        hdr[8] != k.topk || hdr[9] != k.dtype)
+        return 3;
+    const long long cap = ((long long)hdr[11] << 32) | (unsigned int)hdr[10];
+    if (cap != k.cap) return 3;
+    if (hdr[14] != 0) return 4;
+    const long long have = ((long long)hdr[13] << 32) | (unsigned int)hdr[12];
+    return have != k.t ? 1 : 0;
+}
+
+// grid (H, B), 32 threads: one warp scores the new token of one query head.  This is the first kernel of a
+// step: every block compares the header with the call and leaves the state untouched on a mismatch (block
+// (0, 0) records it); the later kernels of the step only look at the status word.
 template <typename T>
 __global__ void step_append_score_kernel(T *__restrict__ kc, T *__restrict__ vc,
                                          float *__restrict__ score, int32_t *__restrict__ hdr,
                                          const T *__restrict__ q, const T *__restrict__ k,
-                                         const T *__restrict__ v, int H, int Hkv, long long cap,
+                                         const T *__restrict__ v, StateKey key, int H, int Hkv, long long cap,
                                          int d, int C, long long t, float scale, float eps) {
     __shared__ float qs[128];
     const int h = blockIdx.x, b = blockIdx.y, rep = H / Hkv, kv = h / rep, lane = threadIdx.x;
-    if (h == 0 && b == 0 && lane == 0) {
-        long long have = ((long long)hdr[13] << 32) | (unsigned int)hdr[12];
-        if (have != t) report_status(hdr + 14, STILL_ERR_STATE_MISMATCH, 1);
+    {
+        const int bad = state_mismatch(hdr, key);
+        if (bad != 0) {
+            if (h == 0 && b == 0 && lane == 0 && bad != 4) report_status(hdr + 14, STILL_ERR_STATE_MISMATCH, bad);
+            return;
+        }
     }
     const T *kn = k + ((long long)b * Hkv + kv) * d;
     T *krow = kc + (((long long)b * Hkv + kv) * cap + t) * d;
@@ -102,9 +128,10 @@ template <typename T>
 __global__ void __launch_bounds__(256)
 step_route_kernel(const T *__restrict__ kc, const T *__restrict__ vc, const float *__restrict__ score,
                   int32_t *__restrict__ sel_idx, uint32_t *__restrict__ sel_mask, float *__restrict__ S,
-                  float *__restrict__ z, const T *__restrict__ Wk, const T *__restrict__ bk, int H, int Hkv, long long cap,
-                  int d, int df, int C, int lam, long long cr) {
+                  float *__restrict__ z, const T *__restrict__ Wk, const T *__restrict__ bk, const int32_t *__restrict__ hdr,
+                  int H, int Hkv, long long cap, int d, int df, int C, int lam, long long cr) {
     extern __shared__ float smem[];
+    if (hdr[14] != 0) return;   // the step's first kernel found the state not to match the call
     const int dp = 2 * df;
     float *ph = smem;                 // [C][dp]
     float *vs = ph + C * dp;          // [C][d]
@@ -174,10 +201,11 @@ template <typename T, int DPL>
 __global__ void __launch_bounds__(128)
 step_attend_kernel(const T *__restrict__ kc, const T *__restrict__ vc,
                    const int32_t *__restrict__ sel_idx, const T *__restrict__ q,
-                   float *__restrict__ part, int H, int Hkv, long long cap, int C, int lam,
-                   long long t, int n_splits, long long cps, long long n_routed, float scale) {
+                   float *__restrict__ part, const int32_t *__restrict__ hdr, int H, int Hkv, long long cap, int C,
+                   int lam, long long t, int n_splits, long long cps, long long n_routed, float scale) {
     constexpr int d = DPL * 32;
     __shared__ float qs[4][d];
+    if (hdr[14] != 0) return;
     const int split = blockIdx.x, kv = blockIdx.y, b = blockIdx.z, rep = H / Hkv;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const T *kh = kc + ((long long)b * Hkv + kv) * cap * d;
@@ -261,6 +289,7 @@ step_merge_kernel(const float *__restrict__ part, const float *__restrict__ S,
                   int32_t *__restrict__ hdr, int H, int d, int df, int n_splits, int la,
                   long long t) {
     __shared__ float qs[128], phi[256], red[4];
+    if (hdr[14] != 0) return;   // mismatch recorded by the step's first kernel: no output, token count unchanged
     const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const long long bh = (long long)b * H + h;
     const int dp = 2 * df;
@@ -342,7 +371,8 @@ static int step_typed(const still_params_t *p, char *state, const still_state_la
     int32_t *hdr = reinterpret_cast<int32_t *>(state + L->header);
     const bool la = lam < C;
 
-    step_append_score_kernel<T><<<dim3(p->H, p->B), 32, 0, st>>>(kc, vc, score, hdr, q, k, v, p->H, p->Hkv,
+    const StateKey key{p->B, p->H, p->Hkv, p->d, p->d_f, p->chunk, p->topk, p->dtype, cap, t};
+    step_append_score_kernel<T><<<dim3(p->H, p->B), 32, 0, st>>>(kc, vc, score, hdr, q, k, v, key, p->H, p->Hkv,
                                                                   cap, d, C, t, p->sm_scale, p->eps);
     ++*launches;
     STILL_CUDA(cudaGetLastError());
@@ -352,7 +382,7 @@ static int step_typed(const still_params_t *p, char *state, const still_state_la
         size_t smem = ((size_t)C * 2 * df + (size_t)C * d + 8 * (size_t)d + C) * 4 + (size_t)C * 4;
         STILL_CUDA(cudaFuncSetAttribute(step_route_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)smem));
-        step_route_kernel<T><<<dim3(p->H, p->B), 256, smem, st>>>(kc, vc, score, sel, smask, S, z, Wk, bk, p->H,
+        step_route_kernel<T><<<dim3(p->H, p->B), 256, smem, st>>>(kc, vc, score, sel, smask, S, z, Wk, bk, hdr, p->H,
                                                                   p->Hkv, cap, d, df, C, lam, c_cur - 2);
         ++*launches;
         STILL_CUDA(cudaGetLastError());
@@ -372,16 +402,14 @@ static int step_typed(const still_params_t *p, char *state, const still_state_la
         // a topk of 0 keeps nothing of the routed chunks: the kernel then sees only the local region
         profile_mark_begin(st);
         if (d == 64) {
-            STILL_CUDA(cudaFuncSetAttribute(step_attend_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            AttendPlan<64>::kTotal));
+            STILL_CUDA(ensure_dynamic_smem((const void *)step_attend_mma_kernel<64>, AttendPlan<64>::kTotal));
             step_attend_mma_kernel<64><<<grid, 128, AttendPlan<64>::kTotal, st>>>(
-                (const __nv_bfloat16 *)kc, (const __nv_bfloat16 *)vc, smask, (const __nv_bfloat16 *)q, part, p->H, p->Hkv,
+                (const __nv_bfloat16 *)kc, (const __nv_bfloat16 *)vc, smask, (const __nv_bfloat16 *)q, part, hdr, p->H, p->Hkv,
                 cap, C, lam, t, n_splits, kMaxSplits + 1, scale_log2);
         } else {
-            STILL_CUDA(cudaFuncSetAttribute(step_attend_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            AttendPlan<128>::kTotal));
+            STILL_CUDA(ensure_dynamic_smem((const void *)step_attend_mma_kernel<128>, AttendPlan<128>::kTotal));
             step_attend_mma_kernel<128><<<grid, 128, AttendPlan<128>::kTotal, st>>>(
-                (const __nv_bfloat16 *)kc, (const __nv_bfloat16 *)vc, smask, (const __nv_bfloat16 *)q, part, p->H, p->Hkv,
+                (const __nv_bfloat16 *)kc, (const __nv_bfloat16 *)vc, smask, (const __nv_bfloat16 *)q, part, hdr, p->H, p->Hkv,
                 cap, C, lam, t, n_splits, kMaxSplits + 1, scale_log2);
         }
         profile_mark_end(st);
@@ -397,10 +425,10 @@ static int step_typed(const still_params_t *p, char *state, const still_state_la
         dim3 grid(n_splits + 1, p->Hkv, p->B);
         profile_mark_begin(st);
         if (d == 64)
-            step_attend_kernel<T, 2><<<grid, 128, 0, st>>>(kc, vc, sel, q, part, p->H, p->Hkv, cap, C, lam, t,
+            step_attend_kernel<T, 2><<<grid, 128, 0, st>>>(kc, vc, sel, q, part, hdr, p->H, p->Hkv, cap, C, lam, t,
                                                            n_splits, cps, n_routed, p->sm_scale);
         else
-            step_attend_kernel<T, 4><<<grid, 128, 0, st>>>(kc, vc, sel, q, part, p->H, p->Hkv, cap, C, lam, t,
+            step_attend_kernel<T, 4><<<grid, 128, 0, st>>>(kc, vc, sel, q, part, hdr, p->H, p->Hkv, cap, C, lam, t,
                                                            n_splits, cps, n_routed, p->sm_scale);
         profile_mark_end(st);
         ++*launches;

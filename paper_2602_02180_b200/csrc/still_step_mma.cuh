@@ -70,10 +70,11 @@ template <int D>
 __global__ void __launch_bounds__(128)
 step_attend_mma_kernel(const __nv_bfloat16 *__restrict__ kc, const __nv_bfloat16 *__restrict__ vc,
                        const uint32_t *__restrict__ sel_mask, const __nv_bfloat16 *__restrict__ q,
-                       float *__restrict__ part, int H, int Hkv, long long cap, int C, int lam, long long t,
-                       int n_splits, int max_splits, float scale_log2) {
+                       float *__restrict__ part, const int32_t *__restrict__ hdr, int H, int Hkv, long long cap, int C,
+                       int lam, long long t, int n_splits, int max_splits, float scale_log2) {
     using P = AttendPlan<D>;
     extern __shared__ __align__(16) uint8_t attend_smem[];
+    if (hdr[14] != 0) return;   // the step's first kernel found the state not to match the call
     uint8_t *smem = attend_smem;
     const int split = blockIdx.x, kv = blockIdx.y, b = blockIdx.z, rep = H / Hkv;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;

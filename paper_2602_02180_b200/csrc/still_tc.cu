@@ -830,6 +830,22 @@ compact_kernel(const __nv_bfloat16 *__restrict__ K, const __nv_bfloat16 *__restr
     }
 }
 
+// The bounded wait of the kernels above, alone: one warp, one mbarrier that expects an arrival which never
+// comes.  No TMA, no tensor memory, no MMA: when the limit has passed the kernel records the timeout and ends.
+__global__ void wait_timeout_selftest_kernel(int *status, long long limit_cycles) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_word;
+    volatile int *abort_flag = &abort_word;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        *abort_flag = 0;
+        fence_barrier_init();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) (void)mbar_wait_limit(&bar, 0, abort_flag, status, 99, limit_cycles);
+    __syncthreads();
+}
+
 // ----------------------------------------------------------------- host side
 
 // 2-D bf16 tensor [rows, d] tiled in boxes of [128 rows, 64 columns] with 128-byte swizzle.
@@ -860,8 +876,7 @@ int launch_tc(const still_params_t *p, long long N, const void *Q, const void *K
         !make_map(&tvs, identity ? V : v_sel, identity ? (unsigned long long)p->B * p->Hkv * N : (unsigned long long)BH * sel_rows, D))
         return STILL_ERR_CUDA;
     const int n_qblocks = (int)((N + 2 * kBlockM - 1) / (2 * kBlockM));
-    if (cudaFuncSetAttribute(sa_merge_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             SmemPlan<D>::kAlloc) != cudaSuccess)
+    if (ensure_dynamic_smem((const void *)sa_merge_tc_kernel<D>, SmemPlan<D>::kAlloc) != cudaSuccess)
         return STILL_ERR_CUDA;
     dim3 grid((unsigned)n_qblocks, (unsigned)BH);
     profile_mark_begin(st);
@@ -883,7 +898,7 @@ int launch_score_tc(const still_params_t *p, long long N, const void *Q, const v
         !make_map(&tk, K, (unsigned long long)p->B * p->Hkv * N, D))
         return STILL_ERR_CUDA;
     constexpr int kSmem = ScoreSmem<D>::kAlloc;
-    if (cudaFuncSetAttribute(score_select_tc_kernel<D, C>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) !=
+    if (ensure_dynamic_smem((const void *)score_select_tc_kernel<D, C>, kSmem) !=
         cudaSuccess)
         return STILL_ERR_CUDA;
     int dev = 0, n_sm = 0;
@@ -909,6 +924,11 @@ int tc_score_select(const still_params_t *p, long long N, const void *Q, const v
     if (p->d == 64 && p->chunk == 128) return launch_score_tc<64, 128>(p, N, Q, K, scores, sel_idx, status_words, st, launches);
     if (p->d == 128 && p->chunk == 64) return launch_score_tc<128, 64>(p, N, Q, K, scores, sel_idx, status_words, st, launches);
     return launch_score_tc<128, 128>(p, N, Q, K, scores, sel_idx, status_words, st, launches);
+}
+
+int tc_selftest_wait_timeout(int *status_words, long long limit_cycles, cudaStream_t st) {
+    wait_timeout_selftest_kernel<<<1, 32, 0, st>>>(status_words, limit_cycles);
+    return cudaGetLastError() == cudaSuccess ? STILL_OK : STILL_ERR_CUDA;
 }
 
 bool tc_supported(const still_params_t *p) {

@@ -9,6 +9,25 @@
 
 namespace still {
 
+// cudaFuncAttributeMaxDynamicSharedMemorySize, set once per kernel and device instead of on every call.
+inline cudaError_t ensure_dynamic_smem(const void *func, int bytes) {
+    struct Done {
+        const void *func;
+        int dev;
+    };
+    constexpr int kSlots = 64;
+    static thread_local Done done[kSlots] = {};
+    static thread_local int n_done = 0;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    for (int i = 0; i < n_done; ++i)
+        if (done[i].func == func && done[i].dev == dev) return cudaSuccess;
+    e = cudaFuncSetAttribute(func, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess && n_done < kSlots) done[n_done++] = Done{func, dev};
+    return e;
+}
+
 // ---- timing of the dominant kernel (still_profile_enable / still_profile_collect) ----
 void profile_mark_begin(cudaStream_t st);
 void profile_mark_end(cudaStream_t st);
@@ -25,6 +44,11 @@ int tc_score_select(const still_params_t *p, long long N, const void *Q, const v
 int tc_sa_merge(const still_params_t *p, long long N, const void *Q, const void *K, const void *V,
                 const int32_t *sel_idx, const float *N_LA, const float *D_LA, void *Y, void *k_sel,
                 void *v_sel, long long sel_rows, int *status_words, cudaStream_t st, int *launches);
+
+// One CTA whose only act is a bounded mbarrier wait on a barrier that nothing arrives on: the wait runs
+// out after limit_cycles, the kernel records STILL_ERR_DEVICE_TIMEOUT (detail 99) in status_words and
+// returns.  Exercises the expiry path of the waits every tcgen05 kernel uses.
+int tc_selftest_wait_timeout(int *status_words, long long limit_cycles, cudaStream_t st);
 
 // ---- tensor-core linear-attention branch of the prefill, bf16 only --------------------
 // True when NP-Map and the chunk-wise state scan of these parameters run on the tcgen05 kernels.

@@ -40,17 +40,17 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Bounded wait.  Returns false (and flags the CTA as aborted) when the limit expires
-// or another role has already aborted.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag,
-                                          int *status, int where) {
+// Bounded wait.  Returns false (and flags the CTA as aborted) when `limit_cycles` have passed
+// or another role has already aborted; `where` goes into the detail word of the status block.
+__device__ __forceinline__ bool mbar_wait_limit(uint64_t *bar, uint32_t parity, volatile int *abort_flag,
+                                                int *status, int where, long long limit_cycles) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     int spins = 0;
     while (!mbar_try_wait(bar, parity)) {
         if ((++spins & 1023) == 0) {
             if (*abort_flag) return false;
-            if (clock64() - t0 > kWaitLimitCycles) {
+            if (clock64() - t0 > limit_cycles) {
                 *abort_flag = 1;
                 report_status(status, STILL_ERR_DEVICE_TIMEOUT, where);
                 return false;
@@ -58,6 +58,10 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
         }
     }
     return true;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag,
+                                          int *status, int where) {
+    return mbar_wait_limit(bar, parity, abort_flag, status, where, kWaitLimitCycles);
 }
 // Bounded wait of the failure path: waits for work already in flight even though the CTA has
 // been flagged as aborted.
@@ -243,8 +247,27 @@ inline EncodeTiledFn encode_fn() {
 
 // 2-D tensor [rows, cols] of 2- or 4-byte elements, tiled in boxes of [box_rows rows, 128 bytes of
 // columns] with 128-byte swizzle (the layout the UMMA descriptors above describe).
+// Encoded maps are kept per host thread (a call encodes the same few maps again and again when a
+// caller reuses its buffers, as a layer does from step to step).
 inline bool make_map_2d(CUtensorMap *m, const void *base, unsigned long long rows, unsigned long long cols,
                         int box_rows, bool fp32) {
+    struct Entry {
+        const void *base;
+        unsigned long long rows, cols;
+        int box_rows, fp32, used;
+        CUtensorMap map;
+    };
+    constexpr int kEntries = 32;
+    static thread_local Entry cache[kEntries] = {};
+    static thread_local int next = 0;
+    for (int i = 0; i < kEntries; ++i) {
+        const Entry &e = cache[i];
+        if (e.used && e.base == base && e.rows == rows && e.cols == cols && e.box_rows == box_rows &&
+            e.fp32 == (int)fp32) {
+            *m = e.map;
+            return true;
+        }
+    }
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     const unsigned esz = fp32 ? 4 : 2;
@@ -252,10 +275,15 @@ inline bool make_map_2d(CUtensorMap *m, const void *base, unsigned long long row
     cuuint64_t strides[1] = {(cuuint64_t)cols * esz};
     cuuint32_t box[2] = {128u / esz, (cuuint32_t)box_rows};
     cuuint32_t estr[2] = {1, 1};
-    return fn(m, fp32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
-              const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    if (fn(m, fp32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+           const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return false;
+    Entry &e = cache[next];
+    next = (next + 1) % kEntries;
+    e = Entry{base, rows, cols, box_rows, (int)fp32, 1, *m};
+    return true;
 }
 
 }  // namespace ptx

@@ -165,8 +165,27 @@ def test_state_full_and_mismatch():
     with pytest.raises(still.StillError) as e:
         still.hybrid_attn_step(p, state, 64, 64, q, k, v, Wq, Wk)
     assert e.value.code == -4
-    # a wrong t_pos is recorded in the state's status word, the context stays usable
+    # a wrong t_pos is recorded in the state's status word; the step writes nothing else (state bytes and y
+    # unchanged), the context stays usable, and later steps on that state are no-ops until it is rebuilt
     state2 = torch.zeros(still.state_bytes(p, 128), dtype=torch.uint8, device="cuda")
     still.hybrid_attn_fwd(p, Q, K, V, Wq, Wk, state=state2, state_max_tokens=128)
-    still.hybrid_attn_step(p, state2, 128, 70, q, k, v, Wq, Wk)
-    assert still.device_status(state2)[0] == -7
+    before = state2.clone()
+    y = torch.full((w.B, w.H, w.d), 7.0, dtype=w.torch_dtype, device="cuda")
+    still.hybrid_attn_step(p, state2, 128, 70, q, k, v, Wq, Wk, y=y)
+    assert still.device_status(state2) == (-7, 1)
+    still.hybrid_attn_step(p, state2, 128, 64, q, k, v, Wq, Wk, y=y)   # the right position, but the state is flagged
+    assert still.device_status(state2) == (-7, 1)
+    same = state2 == before
+    same[14 * 4: 16 * 4] = True    # the status and detail words
+    assert bool(same.all()) and bool((y == 7.0).all())
+    # a state built with other parameters (another topk): detail 3
+    p_other = U.params_of(w.with_(k=4))
+    state3 = torch.zeros(still.state_bytes(p, 128), dtype=torch.uint8, device="cuda")
+    still.hybrid_attn_fwd(p, Q, K, V, Wq, Wk, state=state3, state_max_tokens=128)
+    if still.state_bytes(p_other, 128) <= state3.numel():
+        still.hybrid_attn_step(p_other, state3, 128, 64, q, k, v, Wq, Wk, y=y)
+        assert still.device_status(state3) == (-7, 3)
+    # and the ordinary path still works
+    still.hybrid_attn_fwd(p, Q, K, V, Wq, Wk, state=state2, state_max_tokens=128)
+    still.hybrid_attn_step(p, state2, 128, 64, q, k, v, Wq, Wk, y=y)
+    assert still.device_status(state2) == (0, 0) and torch.isfinite(y.float()).all()

@@ -242,3 +242,19 @@ def test_invalid_arguments_are_rejected():
     with pytest.raises(still.StillError) as e:  # misaligned workspace pointer
         still.hybrid_attn_fwd(p, Q, K, V, Wq, Wk, workspace=ws[1:])
     assert e.value.code == -1
+
+
+def test_bounded_device_wait_runs_out_and_is_reported():
+    # The tensor-core kernels wait on mbarriers with a cycle limit; when a wait runs out the kernel records
+    # STILL_ERR_DEVICE_TIMEOUT in the status block and returns.  The self-test kernel is that wait alone, on a
+    # barrier nothing arrives on, with a limit of about a millisecond: it must come back, report (-6, 99) and
+    # leave the context usable.
+    block = torch.full((256,), 0x5A, dtype=torch.uint8, device="cuda")
+    still.selftest_wait_timeout(block, 2_000_000)
+    assert still.device_status(block) == (-6, 99)
+    w = _small("t", "bf16", 1, 2, 2, 64, 300, 64, 16)
+    r = U.run_prefill(w)
+    assert torch.isfinite(r["Y"].float()).all()
+    ws = torch.empty(still.workspace_bytes(r["p"], w.N), dtype=torch.uint8, device="cuda")
+    still.hybrid_attn_fwd(r["p"], r["Q"], r["K"], r["V"], r["Wq"], r["Wk"], workspace=ws)
+    assert still.device_status(ws) == (0, 0)
