@@ -225,6 +225,8 @@ def main():
     ap.add_argument("--N", type=int, default=None, help="override the sequence length")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-companions", dest="companions", action="store_false",
+                    help="skip the other workloads that the default single-GPU run measures after the headline")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
 
@@ -282,7 +284,18 @@ def _max_over_ranks(torch, dist, x, dev):
     return float(t.item())
 
 
-def bench_prefill(args, w, lam, still, synth, torch, dist, dev, rank, world):
+def roofline_times(work, peaks):
+    """Roofline time of a prefill call: the slower of tensor time and HBM time, with the nominal peaks
+    (2.25 PFLOP/s dense bf16, 8 TB/s) and with this pool's measured ones (burst cuBLAS bf16, copy bandwidth)."""
+    nominal = max(work["flops"] / 2.25e15, work["bytes"] / 8e12)
+    measured = max(work["flops"] / (peaks["bf16_tflops"] * 1e12), work["bytes"] / (peaks["hbm_gbs"] * 1e9))
+    return nominal, measured
+
+
+def time_prefill(w, lam, steps, warmup, still, synth, torch, dist, dev, rank, sample_clocks=True):
+    """Runs warmup + steps prefill calls of workload w with topk lam on resident inputs.  Every timed step
+    has its own CUDA-event pair; the K steps are also bracketed as a whole.  Returns the measurements and
+    the tensors (for the end-to-end leg)."""
     wl = w.with_(k=lam, seed=w.seed + 100 * rank)
     Q, K, V = synth.make_qkv(wl, dev)
     Wq, Wk = synth.make_npmap_weights(wl, dev)
@@ -291,51 +304,92 @@ def bench_prefill(args, w, lam, still, synth, torch, dist, dev, rank, world):
     T = -(-w.N // w.C)
     scores = torch.empty(w.B, w.H, w.N, dtype=torch.float32, device=dev)
     sel = torch.empty(w.B, w.H, T, max(lam, 1), dtype=torch.int32, device=dev)
-    ws = torch.empty(still.workspace_bytes(p, w.N), dtype=torch.uint8, device=dev)
+    ws_bytes = still.workspace_bytes(p, w.N)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
     call = lambda: still.hybrid_attn_fwd(p, Q, K, V, Wq, Wk, Y=Y, scores=scores, sel_idx=sel, workspace=ws)  # noqa: E731
 
-    for _ in range(max(args.warmup, 3)):
+    for _ in range(warmup):
         call()
     launches_per_step = still.last_launch_count()
     _barrier(torch, dist)
     sampler = ClockSampler(dev.index or 0)
-    if rank == 0:
+    if rank == 0 and sample_clocks:
         sampler.start()
-    still.profile_enable(args.steps)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(args.steps):
+    still.profile_enable(steps)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    ev[0].record()
+    for i in range(steps):
         call()
-    e1.record()
+        ev[i + 1].record()
     _barrier(torch, dist)
-    ms_total = e0.elapsed_time(e1)
+    ms_total = ev[0].elapsed_time(ev[-1])
+    per_step = [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
     kernel_ms = still.profile_collect()
-    clocks = sampler.stop() if rank == 0 else None
-    ms_total = _max_over_ranks(torch, dist, ms_total, dev)
+    clocks = sampler.stop() if rank == 0 and sample_clocks else None
     assert still.device_status(ws) == (0, 0), "a device-side wait timed out"
+    return {"ms_total": ms_total, "per_step": per_step, "kernel_ms": kernel_ms, "clocks": clocks,
+            "launches_per_step": launches_per_step, "workspace_bytes": ws_bytes,
+            "tensors": (p, Q, K, V, Wq, Wk)}
+
+
+def prefill_companion(name, w, lam, steps, still, synth, torch, dev):
+    """One more workload in the same run (single GPU): ms per step (median of per-step event pairs), tokens/s
+    and the whole-step fraction of the roofline time, with its own clock sample."""
+    m = time_prefill(w, lam, steps, 3, still, synth, torch, None, dev, 0)
+    del m["tensors"]
+    torch.cuda.empty_cache()
+    work = algorithmic_work(w, lam)
+    peaks = measured_peaks()
+    nominal, measured = roofline_times(work, peaks)
+    ms = statistics.median(m["per_step"])
+    k_ms = statistics.median(m["kernel_ms"]) if m["kernel_ms"] else None
+    out = {"workload": name, "B": w.B, "H": w.H, "Hkv": w.Hkv, "d": w.d, "N": w.N, "chunk": w.C, "topk": lam,
+           "steps": steps, "ms_per_step": ms, "tokens_per_s": w.B * w.N / (ms * 1e-3),
+           "roofline_frac_nominal": nominal / (ms * 1e-3), "roofline_frac_measured": measured / (ms * 1e-3),
+           "workspace_bytes": m["workspace_bytes"], "gpu_launches_per_step": m["launches_per_step"],
+           "clocks": m["clocks"]}
+    if k_ms:
+        ach = work["flops_sa"] / (k_ms * 1e-3) / 1e12
+        out["sa_kernel"] = {"ms": k_ms, "tflops": ach, "frac_of_burst_peak": ach / peaks["bf16_tflops"],
+                            "frac_of_nominal_2250": ach / 2250.0}
+    return out
+
+
+def bench_prefill(args, w, lam, still, synth, torch, dist, dev, rank, world):
+    warmup = max(args.warmup, 10)
+    m = time_prefill(w, lam, args.steps, warmup, still, synth, torch, dist, dev, rank)
+    p, Q, K, V, Wq, Wk = m.pop("tensors")
+    ms_total = _max_over_ranks(torch, dist, m["ms_total"], dev)
+    kernel_ms, clocks, launches_per_step = m["kernel_ms"], m["clocks"], m["launches_per_step"]
     ms_step = ms_total / args.steps
     value = world * w.B * w.N / (ms_step * 1e-3)
 
     work = algorithmic_work(w, lam)
     peaks = measured_peaks()
+    nominal, measured = roofline_times(work, peaks)
     k_ms = statistics.mean(kernel_ms) if kernel_ms else None
     fp32 = w.dtype == "fp32"
     roof = None
     if k_ms:
         ach = work["flops_sa"] / (k_ms * 1e-3) / 1e12
-        peak = peaks["bf16_tflops_sustained"]
+        peak = peaks["bf16_tflops"]
         roof = {"bound": "tensor", "kernel": "softmax-attention + merge", "achieved": ach, "peak": peak,
-                "unit": "TFLOP/s", "frac": ach / peak, "peak_source": peaks["source"] + " (sustained cuBLAS bf16)",
-                "frac_of_burst_peak": ach / peaks["bf16_tflops"], "frac_of_nominal_2250": ach / 2250.0,
-                "kernel_ms": k_ms, "kernel_share_of_step": k_ms / ms_step,
+                "unit": "TFLOP/s", "frac": ach / peak, "peak_source": peaks["source"] + " (burst cuBLAS bf16)",
+                "frac_of_sustained_peak": ach / peaks["bf16_tflops_sustained"], "frac_of_nominal_2250": ach / 2250.0,
+                "kernel_ms": k_ms, "kernel_ms_median": statistics.median(kernel_ms),
+                "kernel_share_of_step": k_ms / ms_step,
                 "traffic": ncu_traffic(f"sa_{w.name}_k{lam}"),
-                "whole_step_frac_of_nominal_roofline": (work["flops"] / 2.25e15) / (ms_step * 1e-3)}
+                "whole_step_frac_of_nominal_roofline": nominal / (ms_step * 1e-3),
+                "whole_step_frac_of_measured_roofline": measured / (ms_step * 1e-3)}
+        if clocks and clocks.get("sm_mhz"):
+            roof["kernel_mcycles_at_sampled_clock"] = k_ms * clocks["sm_mhz"] / 1e3
         if fp32:
             roof["bound"] = "alu"
             roof["note"] = "fp32 inputs run on FMA pipes; peak shown is the bf16 tensor peak for context"
 
     e2e = None
     if not args.no_e2e:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         hQ, hK, hV = (t.cpu().pin_memory() for t in (Q, K, V))
         hWq, hWk = Wq.cpu().pin_memory(), Wk.cpu().pin_memory()
         hY = torch.empty_like(hQ).pin_memory()
@@ -356,6 +410,23 @@ def bench_prefill(args, w, lam, still, synth, torch, dist, dev, rank, world):
         e2e = {"value": world * w.B * w.N / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e, "steps": n_e2e}
         del arena, hQ, hK, hV, hY
+    del Q, K, V
+    torch.cuda.empty_cache()
+
+    # The other workloads, in the same run (single GPU only): every shape once as written and once with a
+    # quarter of each chunk selected, so that selection, NP-Map, state scan and merge run at scale.
+    companions = None
+    if world == 1 and args.companions and args.workload == "c3" and not (args.B or args.H or args.N or args.topk is not None):
+        W = synth.WORKLOADS
+        companions = [
+            prefill_companion("c3 topk=C/4", W["c3"], 16, 5, still, synth, torch, dev),
+            prefill_companion("c2", W["c2"], 64, 10, still, synth, torch, dev),
+            prefill_companion("c2 topk=C/4", W["c2"], 16, 10, still, synth, torch, dev),
+            prefill_companion("c4", W["c4"], 128, 2, still, synth, torch, dev),
+            prefill_companion("c4 topk=C/4", W["c4"], 32, 2, still, synth, torch, dev),
+            decode_companion("c5", W["c5"], 64, 48, still, synth, torch, dev),
+            decode_companion("c5 topk=C/4", W["c5"], 16, 48, still, synth, torch, dev),
+        ]
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -367,34 +438,51 @@ def bench_prefill(args, w, lam, still, synth, torch, dist, dev, rank, world):
 
     return {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "warmup": warmup, "ms_per_step": ms_step, "ms_per_step_median": statistics.median(m["per_step"]),
+        "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16" if not fp32 else "f32", "data": "synthetic",
         "config": {"workload": w.name, "B": w.B, "H": w.H, "Hkv": w.Hkv, "d": w.d, "N": w.N, "chunk": w.C,
-                   "topk": lam, "l2": "inputs larger than L2 (no flush)", "per_gpu_batch": w.B},
+                   "topk": lam, "l2": "inputs larger than L2 (no flush)", "per_gpu_batch": w.B,
+                   "timing": "K steps bracketed by one CUDA-event pair (ms_per_step, value); every step also has its own "
+                             "pair (ms_per_step_median)"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
         "roofline": roof, "cpu_baseline": cpu,
         "algorithmic": {"flops_per_step": work["flops"], "bytes_per_step": work["bytes"]},
+        "workspace_bytes": m["workspace_bytes"], "companions": companions,
     }
 
 
-def bench_decode(args, w, lam, still, synth, torch, dist, dev, rank, world):
-    """c5: the prefix is summarised into a decode state by the prefill, then `steps` decode steps
-    are timed.  HBM-bound: the salient K/V history is read once per KV head per step."""
+def decode_bytes(w, lam, t):
+    """Bytes a decode step at position t has to move: K and V rows of the routed history that at least one
+    query head of the KV group selected (expected size of the union of the group's selections:
+    1 - (1 - lam/C)^group of the rows; all rows when lam = C), read once per KV head, plus the two-chunk local
+    region and, when the linear branch is in use, its state."""
+    rep = w.H // w.Hkv
+    union = 1.0 - (1.0 - lam / w.C) ** rep if lam > 0 else 0.0
+    n_hist = max(t // w.C - 1, 0) * w.C * union
+    return (w.B * w.Hkv * (n_hist + 2 * w.C) * w.d * 2 * 2 +
+            (w.B * w.H * 2 * w.d_f * (w.d + 1) * 4 if lam < w.C else 0))
+
+
+def time_decode(w, lam, n_steps, warmup, still, synth, torch, dist, dev, rank, reserve=0):
+    """Summarises the prefix into a decode state with the prefill, then times n_steps decode steps (one event
+    pair per step and one around all of them)."""
     p = still.StillParams(w.B, w.H, w.Hkv, w.d, w.C, lam, w.torch_dtype)
-    n_steps = args.steps
-    cap = w.N + max(n_steps, w.steps) + args.warmup + 8
-    state = torch.zeros(still.state_bytes(p, cap), dtype=torch.uint8, device=dev)
+    cap = w.N + n_steps + warmup + reserve + 8
+    state_bytes = still.state_bytes(p, cap)
+    state = torch.zeros(state_bytes, dtype=torch.uint8, device=dev)
     Wq, Wk = synth.make_npmap_weights(w, dev)
     wl = w.with_(seed=w.seed + 100 * rank)
     Q, K, V = synth.make_qkv(wl, dev)
     ws = torch.empty(still.workspace_bytes(p, w.N), dtype=torch.uint8, device=dev)
     still.hybrid_attn_fwd(p, Q, K, V, Wq, Wk, state=state, state_max_tokens=cap, workspace=ws, want_y=False)
-    del Q, K, V, ws
     torch.cuda.synchronize()
+    del Q, K, V, ws
+    torch.cuda.empty_cache()
     t = w.N
     ins = [synth.make_decode_inputs(wl, i, dev) for i in range(8)]
     y = torch.empty(w.B, w.H, w.d, dtype=w.torch_dtype, device=dev)
-    for i in range(max(args.warmup, 3)):
+    for i in range(warmup):
         q, k, v = ins[i % 8]
         still.hybrid_attn_step(p, state, cap, t, q, k, v, Wq, Wk, y=y)
         t += 1
@@ -404,33 +492,56 @@ def bench_decode(args, w, lam, still, synth, torch, dist, dev, rank, world):
     if rank == 0:
         sampler.start()
     still.profile_enable(n_steps)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(n_steps + 1)]
+    ev[0].record()
     for i in range(n_steps):
         q, k, v = ins[i % 8]
         still.hybrid_attn_step(p, state, cap, t, q, k, v, Wq, Wk, y=y)
+        ev[i + 1].record()
         t += 1
-    e1.record()
     _barrier(torch, dist)
-    ms_total = _max_over_ranks(torch, dist, e0.elapsed_time(e1), dev)
+    ms_total = ev[0].elapsed_time(ev[-1])
+    per_step = [ev[i].elapsed_time(ev[i + 1]) for i in range(n_steps)]
     kernel_ms = still.profile_collect()
     clocks = sampler.stop() if rank == 0 else None
     assert still.device_status(state)[0] == 0
+    return {"ms_total": ms_total, "per_step": per_step, "kernel_ms": kernel_ms, "clocks": clocks, "launches": launches,
+            "state_bytes": state_bytes, "t": t, "ctx": (p, state, cap, ins, y, Wq, Wk, wl)}
+
+
+def decode_companion(name, w, lam, n_steps, still, synth, torch, dev):
+    m = time_decode(w, lam, n_steps, 3, still, synth, torch, None, dev, 0)
+    del m["ctx"]
+    torch.cuda.empty_cache()
+    peaks = measured_peaks()
+    ms = statistics.median(m["per_step"])
+    by = decode_bytes(w, lam, m["t"])
+    return {"workload": name, "B": w.B, "H": w.H, "Hkv": w.Hkv, "d": w.d, "prefix": w.N, "chunk": w.C, "topk": lam,
+            "steps": n_steps, "ms_per_step": ms, "ms_per_step_max": max(m["per_step"]),
+            "tokens_per_s": w.B / (ms * 1e-3), "algorithmic_bytes_per_step": by,
+            "roofline_frac_nominal": (by / 8e12) / (ms * 1e-3),
+            "roofline_frac_measured": (by / (peaks["hbm_gbs"] * 1e9)) / (ms * 1e-3),
+            "state_bytes": m["state_bytes"], "gpu_launches_per_step": m["launches"], "clocks": m["clocks"]}
+
+
+def bench_decode(args, w, lam, still, synth, torch, dist, dev, rank, world):
+    """c5: the prefix is summarised into a decode state by the prefill, then `steps` decode steps
+    are timed.  HBM-bound: the salient K/V history is read once per KV head per step."""
+    n_steps = args.steps
+    warmup = max(args.warmup, 3)
+    m = time_decode(w, lam, n_steps, warmup, still, synth, torch, dist, dev, rank, reserve=64 + w.steps)
+    p, state, cap, ins, y, Wq, Wk, wl = m.pop("ctx")
+    t, launches, clocks, kernel_ms = m["t"], m["launches"], m["clocks"], m["kernel_ms"]
+    ms_total = _max_over_ranks(torch, dist, m["ms_total"], dev)
     ms_step = ms_total / n_steps
     peaks = measured_peaks()
-    es = 2
-    # K and V rows of the routed history that at least one query head of the KV group selected (expected
-    # size of the union of the group's selections: 1 - (1 - lam/C)^group of the rows; all rows when
-    # lam = C), read once per KV head, plus the local region and, when it is in use, the LA state
-    rep = w.H // w.Hkv
-    union = 1.0 - (1.0 - lam / w.C) ** rep if lam > 0 else 0.0
-    n_hist = (t // w.C - 1) * w.C * union
-    by = w.B * w.Hkv * (n_hist + 2 * w.C) * w.d * es * 2 + (w.B * w.H * 2 * w.d_f * (w.d + 1) * 4 if lam < w.C else 0)
+    by = decode_bytes(w, lam, t)
     k_ms = statistics.mean(kernel_ms) if kernel_ms else ms_step
     ach = by / (k_ms * 1e-3) / 1e9
     roof = {"bound": "hbm", "kernel": "split-KV attend", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
             "frac": ach / peaks["hbm_gbs"], "peak_source": peaks["source"], "kernel_ms": k_ms,
             "traffic": ncu_traffic(f"attend_{w.name}_k{lam}")}
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     # end to end: every step copies that step's q, k, v from pinned host memory and reads y back
     e2e = None
     if not args.no_e2e:
@@ -464,7 +575,8 @@ def bench_decode(args, w, lam, still, synth, torch, dist, dev, rank, world):
 
     return {
         "metric": "hybrid-attn decode tokens/s/layer at Llama-3-8B shape", "value": world * w.B / (ms_step * 1e-3),
-        "unit": UNIT, "n_gpus": world, "steps": n_steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_step,
+        "unit": UNIT, "n_gpus": world, "steps": n_steps, "warmup": warmup, "ms_per_step": ms_step,
+        "ms_per_step_median": statistics.median(m["per_step"]),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": w.name, "B": w.B, "H": w.H, "Hkv": w.Hkv, "d": w.d, "prefix": w.N, "chunk": w.C,
                    "topk": lam, "l2": "K/V history larger than L2 (no flush)"},

@@ -98,6 +98,218 @@ __device__ __forceinline__ int sel_limit(long long pos, int C, int lam) {  // vi
     return c >= 2 ? (int)((c - 1) * lam) : 0;
 }
 
+// ---------------------------------------------------------------------------
+// Softmax warps of the attention kernels (one warpgroup per query tile, a thread per query row) and the
+// merge epilogue.  `st` describes the CTA's (or the CTA pair's) key stream, x is the query tile (0: A, 1: B),
+// tile_row0 the position of the tile's first row, stage_tile the tile's Q region in shared memory (the
+// epilogue's staging space).  The barriers are this CTA's, except that in a CTA pair the two halves of P
+// are announced on the first CTA's p_half barriers (p_half_cluster: their address in the cluster window).
+// ---------------------------------------------------------------------------
+template <int D, int kKStages, int kVStages, bool kPair, class StreamT>
+__device__ __forceinline__ void softmax_role(const StreamT &st, const int x, const int tile_row0, const uint32_t tmem_base,
+                                             uint64_t *s_full, uint64_t *k_empty, uint64_t *v_empty, uint64_t *p_half,
+                                             const uint32_t p_half_cluster, uint64_t *o_final, volatile int *abort_flag,
+                                             int *status, uint8_t *stage_tile, const float *__restrict__ N_LA,
+                                             const float *__restrict__ D_LA, __nv_bfloat16 *__restrict__ Y, const int bh,
+                                             const int N, const int C, const int lam, const float scale_log2) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    auto col_s = [](int xx) -> uint32_t { return (uint32_t)xx * 128u; };
+    auto col_o = [](int xx) -> uint32_t { return 256u + (uint32_t)xx * (uint32_t)D; };
+    auto arrive_p = [&](int half) {
+        if constexpr (kPair) mbar_arrive_cluster(p_half_cluster + (uint32_t)(2 * x + half) * 8u);
+        else mbar_arrive(p_half + 2 * x + half);
+    };
+        const int row_in_tile = ((warp & 3) << 5) | lane;
+    const int t = tile_row0 + row_in_tile;         // this thread's query position
+    const bool tile_present = (x == 0) || st.has_b;   // (a tile without rows below N still runs in a pair)
+    if (tile_present) {
+        const uint32_t lane_addr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+        const int tq = min(t, N - 1);              // rows past N mimic the last row (never stored)
+        const int c = tq / C;
+        const int lim_sel = c >= 2 ? (c - 1) * lam : 0;
+        const int loc_lo = c >= 1 ? (c - 1) * C : 0;
+        float m_used = -INFINITY, l_sum = 0.f;     // log2 domain
+        int n_seen = 0, prev_i = -1;
+        bool ok = true;
+        for (int i = 0; i < st.n_tiles && ok; ++i) {
+            if (!st.used_by(x, i)) continue;
+            // visible column interval [lo, hi] of this row in stream tile i
+            int lo, hi;
+            if (st.is_sel(i)) {
+                lo = 0;
+                hi = lim_sel - i * kBlockN - 1;
+            } else {
+                const int p0 = st.loc_m(i) * kBlockN;
+                lo = loc_lo - p0;
+                hi = tq - p0;
+            }
+            lo = max(lo, 0);
+            hi = min(hi, kBlockN - 1);
+            const bool need_mask = __any_sync(0xffffffffu, lo > 0 || hi < kBlockN - 1);
+            ok = mbar_wait(s_full + x, n_seen & 1, abort_flag, status, 8);
+            if (!ok) break;
+            tc_fence_after();
+            if (row_in_tile == 0) {
+                // S_x of tile i is complete, and so is everything the MMA warp issued before it (each
+                // tcgen05.commit costs the tensor pipe a bubble, so the ring stages are released here
+                // instead): tile x is done with this K stage and with the V stage of its previous tile.
+                mbar_arrive(k_empty + i % kKStages);
+                if (prev_i >= 0) mbar_arrive(v_empty + prev_i % kVStages);
+            }
+            prev_i = i;
+            uint32_t sr[128];
+            tmem_ld32(lane_addr + col_s(x) + 0, sr + 0);
+            tmem_ld32(lane_addr + col_s(x) + 32, sr + 32);
+            tmem_ld32(lane_addr + col_s(x) + 64, sr + 64);
+            tmem_ld32(lane_addr + col_s(x) + 96, sr + 96);
+            tmem_wait_ld();
+            float *s = reinterpret_cast<float *>(sr);
+            if (need_mask) {
+#pragma unroll
+                for (int j = 0; j < 128; ++j)
+                    if (j < lo || j > hi) s[j] = -INFINITY;
+            }
+            float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < 128; j += 8) {
+                mx0 = max3(mx0, s[j], s[j + 1]);
+                mx1 = max3(mx1, s[j + 2], s[j + 3]);
+                mx2 = max3(mx2, s[j + 4], s[j + 5]);
+                mx3 = max3(mx3, s[j + 6], s[j + 7]);
+            }
+            const float mt = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * scale_log2;
+            // lazy rescale: keep the old reference unless the new maximum exceeds it by 2^8
+            const bool grow = mt > m_used + 8.f;
+            float alpha = 1.f;
+            if (grow) {
+                alpha = (m_used == -INFINITY) ? 0.f : ex2(m_used - mt);
+                m_used = mt;
+            }
+            if (n_seen > 0 && __any_sync(0xffffffffu, grow)) {
+                // S of this tile was committed after the previous P V product: O is quiescent
+#pragma unroll
+                for (int q = 0; q < D / 32; ++q) {
+                    uint32_t orow[32];
+                    tmem_ld32(lane_addr + col_o(x) + q * 32, orow);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) orow[j] = __float_as_uint(__uint_as_float(orow[j]) * alpha);
+                    tmem_st32(lane_addr + col_o(x) + q * 32, orow);
+                }
+            }
+            l_sum *= alpha;
+            const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
+            const float2 scale2 = make_float2(scale_log2, scale_log2), negm2 = make_float2(neg_m, neg_m);
+            float2 acc = make_float2(0.f, 0.f);
+            // P = 2^(s * scale - m) as bf16 over S, in two halves of 64 columns; the MMA warp
+            // starts on the first half while the second is computed.  (All exponentials go to the
+            // MUFU unit: with a cubic 2^x on the FMA pipes for a quarter, half or three quarters of them the
+            // kernel was measured 3.6 % slower per quarter -- every added instruction of this warp costs about a
+            // cycle of the tile's serial chain.)
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                uint32_t pk[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    const float2 sv = make_float2(s[q * 64 + 2 * j], s[q * 64 + 2 * j + 1]);
+                    const float2 xv = __ffma2_rn(sv, scale2, negm2);
+                    const float2 pr = make_float2(ex2(xv.x), ex2(xv.y));
+                    acc = __fadd2_rn(acc, pr);
+                    pk[j] = pack_bf16(pr.x, pr.y);
+                    if (q == 1 && j == 12) {
+                        // the first half of P has had time to land: hand it to the MMA warp
+                        tmem_wait_st();
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) arrive_p(0);
+                    }
+                }
+                tmem_st32(lane_addr + col_s(x) + q * 32, pk);
+            }
+            l_sum += acc.x + acc.y;
+            tmem_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) arrive_p(1);
+            ++n_seen;
+        }
+        // ---- epilogue: y = (O e^{m-ms} + e^{-ms} N_LA) / (l e^{m-ms} + e^{-ms} D_LA), ms = max(m, 0)
+        // A thread owns a row, but loads / stores in which every lane touches a different row cost a
+        // memory instruction per 16 bytes and row; so N_LA comes in and Y goes out through shared memory
+        // with 16 consecutive lanes per row.  The staging space is this warp's 32 rows of the tile's Q
+        // region (one row = D bf16 = 2 D bytes), free once the tile's last Q K^T has completed; 16-byte
+        // pieces are swizzled by the row so that row-wise and piece-wise accesses avoid bank conflicts.
+        if (ok) ok = mbar_wait(o_final + x, 0, abort_flag, status, 9);
+        ok = __all_sync(0xffffffffu, ok);
+        if (ok) {
+            tc_fence_after();
+            constexpr int kRowBytes = D * 2, kPieces = kRowBytes / 16;   // pieces of 16 bytes per staged row
+            uint8_t *stg = stage_tile + (warp & 3) * 32 * kRowBytes;
+            const int t0 = tile_row0 + (warp & 3) * 32;                    // first row of this warp
+            float fs = 1.f, fl = 0.f, dla = 0.f;
+            if (D_LA != nullptr && t < N) {
+                dla = D_LA[(long long)bh * N + t];
+                if (dla > 0.f) {
+                    const float m_nat = m_used * 0.6931471805599453f;
+                    const float ms = fmaxf(m_nat, 0.f);
+                    fs = __expf(m_nat - ms);
+                    fl = __expf(-ms);
+                }
+            }
+            const float inv = 1.f / (l_sum * fs + fl * dla);
+            const bool with_la = (D_LA != nullptr) && __any_sync(0xffffffffu, dla > 0.f);
+            uint32_t out[D / 2];   // the row as packed bf16
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {   // halves of D / 2 columns: as fp32 they fill one staged row
+                if (with_la) {
+                    __syncwarp();
+#pragma unroll
+                    for (int it = 0; it < kPieces; ++it) {
+                        const int id = it * 32 + lane, row = id / kPieces, c = id % kPieces;
+                        uint4 v = make_uint4(0, 0, 0, 0);
+                        if (t0 + row < N)
+                            v = *reinterpret_cast<const uint4 *>(N_LA + ((long long)bh * N + t0 + row) * D + hh * (D / 2) + c * 4);
+                        *reinterpret_cast<uint4 *>(stg + row * kRowBytes + ((c ^ (row & (kPieces - 1))) << 4)) = v;
+                    }
+                    __syncwarp();
+                }
+#pragma unroll
+                for (int q = 0; q < D / 64; ++q) {
+                    uint32_t orow[32];
+                    tmem_ld32(lane_addr + col_o(x) + hh * (D / 2) + q * 32, orow);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int j4 = 0; j4 < 8; ++j4) {
+                        float4 nl = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (with_la)
+                            nl = *reinterpret_cast<const float4 *>(stg + lane * kRowBytes + (((q * 8 + j4) ^ (lane & (kPieces - 1))) << 4));
+                        const float a0 = fmaf(fl, nl.x, __uint_as_float(orow[4 * j4]) * fs);
+                        const float a1 = fmaf(fl, nl.y, __uint_as_float(orow[4 * j4 + 1]) * fs);
+                        const float a2 = fmaf(fl, nl.z, __uint_as_float(orow[4 * j4 + 2]) * fs);
+                        const float a3 = fmaf(fl, nl.w, __uint_as_float(orow[4 * j4 + 3]) * fs);
+                        out[hh * (D / 4) + q * 16 + 2 * j4] = pack_bf16(a0 * inv, a1 * inv);
+                        out[hh * (D / 4) + q * 16 + 2 * j4 + 1] = pack_bf16(a2 * inv, a3 * inv);
+                    }
+                }
+            }
+            // Y: own row into the staging space, then the warp writes its 32 rows piece-wise
+            __syncwarp();
+#pragma unroll
+            for (int c = 0; c < kPieces; ++c)
+                *reinterpret_cast<uint4 *>(stg + lane * kRowBytes + ((c ^ (lane & (kPieces - 1))) << 4)) =
+                    make_uint4(out[4 * c], out[4 * c + 1], out[4 * c + 2], out[4 * c + 3]);
+            __syncwarp();
+#pragma unroll
+            for (int it = 0; it < kPieces; ++it) {
+                const int id = it * 32 + lane, row = id / kPieces, c = id % kPieces;
+                if (t0 + row < N)
+                    *reinterpret_cast<uint4 *>(Y + ((long long)bh * N + t0 + row) * D + c * 8) =
+                        *reinterpret_cast<const uint4 *>(stg + row * kRowBytes + ((c ^ (row & (kPieces - 1))) << 4));
+            }
+        }
+    }
+}
+
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -316,200 +528,311 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         reg_inc<216>();
         // ------------------------------------------------------------ softmax + epilogue
         const int x = (warp - 4) >> 2;                 // 0: tile A, 1: tile B
-        const int row_in_tile = ((warp & 3) << 5) | lane;
-        const int t = R0 + x * kBlockM + row_in_tile;  // this thread's query position
-        const bool tile_present = (x == 0) || st.has_b;
-        if (tile_present) {
-            const uint32_t lane_addr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
-            const int tq = min(t, N - 1);              // rows past N mimic the last row (never stored)
-            const int c = tq / C;
-            const int lim_sel = c >= 2 ? (c - 1) * lam : 0;
-            const int loc_lo = c >= 1 ? (c - 1) * C : 0;
-            float m_used = -INFINITY, l_sum = 0.f;     // log2 domain
-            int n_seen = 0, prev_i = -1;
-            bool ok = true;
-            for (int i = 0; i < st.n_tiles && ok; ++i) {
-                if (!st.used_by(x, i)) continue;
-                // visible column interval [lo, hi] of this row in stream tile i
-                int lo, hi;
-                if (st.is_sel(i)) {
-                    lo = 0;
-                    hi = lim_sel - i * kBlockN - 1;
-                } else {
-                    const int p0 = st.loc_m(i) * kBlockN;
-                    lo = loc_lo - p0;
-                    hi = tq - p0;
-                }
-                lo = max(lo, 0);
-                hi = min(hi, kBlockN - 1);
-                const bool need_mask = __any_sync(0xffffffffu, lo > 0 || hi < kBlockN - 1);
-                ok = mbar_wait(s_full + x, n_seen & 1, abort_flag, status, 8);
-                if (!ok) break;
-                tc_fence_after();
-                if (row_in_tile == 0) {
-                    // S_x of tile i is complete, and so is everything the MMA warp issued before it (each
-                    // tcgen05.commit costs the tensor pipe a bubble, so the ring stages are released here
-                    // instead): tile x is done with this K stage and with the V stage of its previous tile.
-                    mbar_arrive(k_empty + i % P::kKStages);
-                    if (prev_i >= 0) mbar_arrive(v_empty + prev_i % P::kVStages);
-                }
-                prev_i = i;
-                uint32_t sr[128];
-                tmem_ld32(lane_addr + col_s(x) + 0, sr + 0);
-                tmem_ld32(lane_addr + col_s(x) + 32, sr + 32);
-                tmem_ld32(lane_addr + col_s(x) + 64, sr + 64);
-                tmem_ld32(lane_addr + col_s(x) + 96, sr + 96);
-                tmem_wait_ld();
-                float *s = reinterpret_cast<float *>(sr);
-                if (need_mask) {
-#pragma unroll
-                    for (int j = 0; j < 128; ++j)
-                        if (j < lo || j > hi) s[j] = -INFINITY;
-                }
-                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-#pragma unroll
-                for (int j = 0; j < 128; j += 8) {
-                    mx0 = max3(mx0, s[j], s[j + 1]);
-                    mx1 = max3(mx1, s[j + 2], s[j + 3]);
-                    mx2 = max3(mx2, s[j + 4], s[j + 5]);
-                    mx3 = max3(mx3, s[j + 6], s[j + 7]);
-                }
-                const float mt = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * scale_log2;
-                // lazy rescale: keep the old reference unless the new maximum exceeds it by 2^8
-                const bool grow = mt > m_used + 8.f;
-                float alpha = 1.f;
-                if (grow) {
-                    alpha = (m_used == -INFINITY) ? 0.f : ex2(m_used - mt);
-                    m_used = mt;
-                }
-                if (n_seen > 0 && __any_sync(0xffffffffu, grow)) {
-                    // S of this tile was committed after the previous P V product: O is quiescent
-#pragma unroll
-                    for (int q = 0; q < D / 32; ++q) {
-                        uint32_t orow[32];
-                        tmem_ld32(lane_addr + col_o(x) + q * 32, orow);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) orow[j] = __float_as_uint(__uint_as_float(orow[j]) * alpha);
-                        tmem_st32(lane_addr + col_o(x) + q * 32, orow);
-                    }
-                }
-                l_sum *= alpha;
-                const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
-                const float2 scale2 = make_float2(scale_log2, scale_log2), negm2 = make_float2(neg_m, neg_m);
-                float2 acc = make_float2(0.f, 0.f);
-                // P = 2^(s * scale - m) as bf16 over S, in two halves of 64 columns; the MMA warp
-                // starts on the first half while the second is computed.  (All exponentials go to the
-                // MUFU unit: a Cody-Waite / cubic 2^x on the FMA pipes was measured and costs more
-                // issue slots and FMA-pipe cycles per element than MUFU does.)
-#pragma unroll
-                for (int q = 0; q < 2; ++q) {
-                    uint32_t pk[32];
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const float2 sv = make_float2(s[q * 64 + 2 * j], s[q * 64 + 2 * j + 1]);
-                        const float2 xv = __ffma2_rn(sv, scale2, negm2);
-                        const float2 pr = make_float2(ex2(xv.x), ex2(xv.y));
-                        acc = __fadd2_rn(acc, pr);
-                        pk[j] = pack_bf16(pr.x, pr.y);
-                        if (q == 1 && j == 12) {
-                            // the first half of P has had time to land: hand it to the MMA warp
-                            tmem_wait_st();
-                            tc_fence_before();
-                            __syncwarp();
-                            if (lane == 0) mbar_arrive(p_half + 2 * x);
-                        }
-                    }
-                    tmem_st32(lane_addr + col_s(x) + q * 32, pk);
-                }
-                l_sum += acc.x + acc.y;
-                tmem_wait_st();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(p_half + 2 * x + 1);
-                ++n_seen;
-            }
-            // ---- epilogue: y = (O e^{m-ms} + e^{-ms} N_LA) / (l e^{m-ms} + e^{-ms} D_LA), ms = max(m, 0)
-            // A thread owns a row, but loads / stores in which every lane touches a different row cost a
-            // memory instruction per 16 bytes and row; so N_LA comes in and Y goes out through shared memory
-            // with 16 consecutive lanes per row.  The staging space is this warp's 32 rows of the tile's Q
-            // region (one row = D bf16 = 2 D bytes), free once the tile's last Q K^T has completed; 16-byte
-            // pieces are swizzled by the row so that row-wise and piece-wise accesses avoid bank conflicts.
-            if (ok) ok = mbar_wait(o_final + x, 0, abort_flag, status, 9);
-            ok = __all_sync(0xffffffffu, ok);
-            if (ok) {
-                tc_fence_after();
-                constexpr int kRowBytes = D * 2, kPieces = kRowBytes / 16;   // pieces of 16 bytes per staged row
-                uint8_t *stg = smem + P::kQ + x * P::kTileBytes + (warp & 3) * 32 * kRowBytes;
-                const int t0 = R0 + x * kBlockM + (warp & 3) * 32;           // first row of this warp
-                float fs = 1.f, fl = 0.f, dla = 0.f;
-                if (D_LA != nullptr && t < N) {
-                    dla = D_LA[(long long)bh * N + t];
-                    if (dla > 0.f) {
-                        const float m_nat = m_used * 0.6931471805599453f;
-                        const float ms = fmaxf(m_nat, 0.f);
-                        fs = __expf(m_nat - ms);
-                        fl = __expf(-ms);
-                    }
-                }
-                const float inv = 1.f / (l_sum * fs + fl * dla);
-                const bool with_la = (D_LA != nullptr) && __any_sync(0xffffffffu, dla > 0.f);
-                uint32_t out[D / 2];   // the row as packed bf16
-#pragma unroll
-                for (int hh = 0; hh < 2; ++hh) {   // halves of D / 2 columns: as fp32 they fill one staged row
-                    if (with_la) {
-                        __syncwarp();
-#pragma unroll
-                        for (int it = 0; it < kPieces; ++it) {
-                            const int id = it * 32 + lane, row = id / kPieces, c = id % kPieces;
-                            uint4 v = make_uint4(0, 0, 0, 0);
-                            if (t0 + row < N)
-                                v = *reinterpret_cast<const uint4 *>(N_LA + ((long long)bh * N + t0 + row) * D + hh * (D / 2) + c * 4);
-                            *reinterpret_cast<uint4 *>(stg + row * kRowBytes + ((c ^ (row & (kPieces - 1))) << 4)) = v;
-                        }
-                        __syncwarp();
-                    }
-#pragma unroll
-                    for (int q = 0; q < D / 64; ++q) {
-                        uint32_t orow[32];
-                        tmem_ld32(lane_addr + col_o(x) + hh * (D / 2) + q * 32, orow);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int j4 = 0; j4 < 8; ++j4) {
-                            float4 nl = make_float4(0.f, 0.f, 0.f, 0.f);
-                            if (with_la)
-                                nl = *reinterpret_cast<const float4 *>(stg + lane * kRowBytes + (((q * 8 + j4) ^ (lane & (kPieces - 1))) << 4));
-                            const float a0 = fmaf(fl, nl.x, __uint_as_float(orow[4 * j4]) * fs);
-                            const float a1 = fmaf(fl, nl.y, __uint_as_float(orow[4 * j4 + 1]) * fs);
-                            const float a2 = fmaf(fl, nl.z, __uint_as_float(orow[4 * j4 + 2]) * fs);
-                            const float a3 = fmaf(fl, nl.w, __uint_as_float(orow[4 * j4 + 3]) * fs);
-                            out[hh * (D / 4) + q * 16 + 2 * j4] = pack_bf16(a0 * inv, a1 * inv);
-                            out[hh * (D / 4) + q * 16 + 2 * j4 + 1] = pack_bf16(a2 * inv, a3 * inv);
-                        }
-                    }
-                }
-                // Y: own row into the staging space, then the warp writes its 32 rows piece-wise
-                __syncwarp();
-#pragma unroll
-                for (int c = 0; c < kPieces; ++c)
-                    *reinterpret_cast<uint4 *>(stg + lane * kRowBytes + ((c ^ (lane & (kPieces - 1))) << 4)) =
-                        make_uint4(out[4 * c], out[4 * c + 1], out[4 * c + 2], out[4 * c + 3]);
-                __syncwarp();
-#pragma unroll
-                for (int it = 0; it < kPieces; ++it) {
-                    const int id = it * 32 + lane, row = id / kPieces, c = id % kPieces;
-                    if (t0 + row < N)
-                        *reinterpret_cast<uint4 *>(Y + ((long long)bh * N + t0 + row) * D + c * 8) =
-                            *reinterpret_cast<const uint4 *>(stg + row * kRowBytes + ((c ^ (row & (kPieces - 1))) << 4));
-                }
-            }
-        }
+        softmax_role<D, P::kKStages, P::kVStages, false>(st, x, R0 + x * kBlockM, tmem_base, s_full, k_empty, v_empty, p_half, 0u,
+                                                         o_final, abort_flag, status, smem + P::kQ + x * P::kTileBytes, N_LA,
+                                                         D_LA, Y, bh, N, C, lam, scale_log2);
     }
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, 512);
+    }
+}
+
+// ---------------------------------------------------------------------------
+// The same branch on CTA pairs (head dim 128): two CTAs of a cluster work on 512 consecutive query rows of
+// one (batch, head) with UMMAs of the cta_group::2 form.  Query tile X of the pair is 256 rows -- rows
+// [R0 + 256 X + 128 r, + 128) belong to the CTA of cluster rank r -- and one instruction, issued by a thread
+// of rank 0, computes S_X = Q_X K^T (or O_X += P_X V) for both CTAs.  Each CTA keeps only its half of every
+// key tile in shared memory: 64 of the 128 keys of K (the B operand of Q K^T is split along N) and 64 of the
+// 128 value columns of V (likewise for P V); the tensor cores of both SMs read both halves.  Per FLOP a CTA
+// therefore pulls half the K / V bytes from L2 and reads a quarter less shared memory than a CTA working
+// alone, and the rings hold five stages each.
+//
+// Who signals whom.  K / V / Q tiles: every CTA loads its halves into its own shared memory with plain TMA
+// loads (no multicast) whose byte counts complete on the full-barriers of rank 0, where the issuing thread
+// waits.  S_X ready, O_X final: one tcgen05.commit arrives on the barrier of both CTAs.  P_X written: the
+// softmax warps of both CTAs arrive on rank 0's p_half barriers (eight arrivals).  Ring stages are released
+// locally: when a CTA's softmax warps see S_X of stream tile i, the pair's instruction has completed in both
+// CTAs.  Everything else -- stream, masks, online softmax, merge epilogue -- is as in the kernel above.
+// ---------------------------------------------------------------------------
+template <int D>
+struct PairPlan {
+    static constexpr int kQTile = kBlockM * D * 2;             // one Q tile of this CTA (128 rows)
+    static constexpr int kKHalf = (kBlockN / 2) * D * 2;       // 64 keys of a K tile
+    static constexpr int kVHalf = kBlockN * (D / 2) * 2;       // 128 keys x D / 2 value columns
+    static constexpr int kKStages = 5, kVStages = 5;
+    static constexpr int kQ = 0;
+    static constexpr int kK = kQ + 2 * kQTile;
+    static constexpr int kV = kK + kKStages * kKHalf;
+    static constexpr int kBar = kV + kVStages * kVHalf;
+    static constexpr int kNumBars = 1 + 2 * kKStages + 2 * kVStages + 9;
+    static constexpr int kMisc = kBar + kNumBars * 8;          // tmem base, abort flag, "a CTA has failed before"
+    static constexpr int kTotal = kMisc + 16;
+    static constexpr int kAlloc = kTotal + 1024;
+};
+static_assert(PairPlan<128>::kAlloc <= kMaxDynamicSmem, "pair attention kernel: the shared-memory plan exceeds what a CTA can have");
+
+// Key stream of a CTA pair (same in both CTAs): SEL tiles, then the LOC tiles m_first .. m_last.
+struct PairStream {
+    int n_sel_a, n_sel_b, m0, m_first, has_b, n_tiles;
+    __device__ __forceinline__ bool is_sel(int i) const { return i < n_sel_b; }
+    __device__ __forceinline__ int loc_m(int i) const { return m_first + (i - n_sel_b); }
+    __device__ __forceinline__ bool used_by(int x, int i) const {
+        if (i < n_sel_b) return x == 0 ? (i < n_sel_a) : true;
+        const int m = loc_m(i);
+        return x == 0 ? (m <= m0 + 1) : (m >= m0 + 1);
+    }
+};
+
+template <int D>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+sa_merge_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                     const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_ksel,
+                     const __grid_constant__ CUtensorMap tm_vsel, const float *__restrict__ N_LA,
+                     const float *__restrict__ D_LA, __nv_bfloat16 *__restrict__ Y, int *status, int H, int Hkv, int N,
+                     int C, int lam, int sel_rows, int sel_identity, float scale_log2, int n_pairs) {
+    using P = PairPlan<D>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + P::kBar);
+    uint64_t *q_full = bars;
+    uint64_t *k_full = bars + 1, *k_empty = k_full + P::kKStages;
+    uint64_t *v_full = k_empty + P::kKStages, *v_empty = v_full + P::kVStages;
+    uint64_t *s_full = v_empty + P::kVStages;  // [2]
+    uint64_t *p_half = s_full + 2;             // [2][2]
+    uint64_t *o_final = p_half + 4;            // [2]
+    uint64_t *drain = o_final + 2;
+    uint32_t *tmem_base_slot = reinterpret_cast<uint32_t *>(smem + P::kMisc);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + P::kMisc + 4);
+    volatile int *failed_before = reinterpret_cast<volatile int *>(smem + P::kMisc + 8);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank(), peer = rank ^ 1u;
+    const int pb = n_pairs - 1 - (int)(blockIdx.x >> 1);  // heavy blocks first
+    const int bh = blockIdx.y, b = bh / H, h = bh % H, kvh = h / (H / Hkv);
+    const int R0 = pb * 4 * kBlockM;
+
+    PairStream st;
+    st.m0 = R0 / kBlockN;
+    st.m_first = st.m0 - (st.m0 > 0 ? 1 : 0);
+    st.has_b = (R0 + 2 * kBlockM) < N;
+    {
+        const int last_a = min(R0 + 2 * kBlockM - 1, N - 1), last_b = min(R0 + 4 * kBlockM - 1, N - 1);
+        st.n_sel_a = (sel_limit(last_a, C, lam) + kBlockN - 1) / kBlockN;
+        st.n_sel_b = st.has_b ? (sel_limit(last_b, C, lam) + kBlockN - 1) / kBlockN : st.n_sel_a;
+        const int m_last = min(st.m0 + (st.has_b ? 3 : 1), (N - 1) / kBlockN);
+        st.n_tiles = st.n_sel_b + (m_last - st.m_first + 1);
+    }
+
+    if (threadIdx.x == 0) {
+        mbar_init(q_full, 1);
+        for (int i = 0; i < P::kKStages; ++i) { mbar_init(k_full + i, 1); mbar_init(k_empty + i, 2); }
+        for (int i = 0; i < P::kVStages; ++i) { mbar_init(v_full + i, 1); mbar_init(v_empty + i, 2); }
+        for (int i = 0; i < 2; ++i) { mbar_init(s_full + i, 1); mbar_init(o_final + i, 1); }
+        for (int i = 0; i < 4; ++i) mbar_init(p_half + i, 8);  // one arrival per softmax warp of either CTA
+        mbar_init(drain, 1);
+        *abort_flag = 0;
+        *failed_before = 0;
+        fence_barrier_init();
+    }
+    // The peer's barriers exist and its shared memory may be written from here on.
+    cluster_sync_all();
+    // A pair that starts after some CTA has reported a failure does nothing; rank 0 decides for both.
+    if (threadIdx.x == 0 && rank == 0) {
+        const int seen = *reinterpret_cast<volatile int *>(status) != 0;
+        *failed_before = seen;
+        st_cluster_u32(mapa(smem_u32(const_cast<int *>(failed_before)), 1), (uint32_t)seen);
+    }
+    cluster_sync_all();
+    if (*failed_before) return;
+    if (warp == 1) {
+        tmem_alloc_pair(tmem_base_slot, 512);
+        tmem_relinquish_pair();
+    }
+    tc_fence_before();
+    cluster_sync_all();   // both CTAs hold their tensor memory before the first instruction of the pair
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_base_slot;
+    auto col_s = [](int x) -> uint32_t { return (uint32_t)x * 128u; };
+    auto col_o = [](int x) -> uint32_t { return 256u + (uint32_t)x * (uint32_t)D; };
+    // a role that gives up tells the other CTA, whose waits would otherwise run to their own limit
+    auto tell_peer = [&]() { st_cluster_u32(mapa(smem_u32(const_cast<int *>(abort_flag)), peer), 1u); };
+
+    if (warp < 4) {
+    reg_dec<72>();
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer (both CTAs)
+        if (lane == 0) {
+            const uint32_t q_full0 = mapa(smem_u32(q_full), 0), k_full0 = mapa(smem_u32(k_full), 0),
+                           v_full0 = mapa(smem_u32(v_full), 0);
+            const int n_q = st.has_b ? 2 : 1;
+            const int q_row = bh * N + R0 + (int)rank * kBlockM;
+            if (rank == 0) mbar_expect_tx(q_full, 2 * n_q * P::kQTile);   // both CTAs' tiles
+            for (int x = 0; x < n_q; ++x)
+                for (int half = 0; half < D / 64; ++half)
+                    tma_load_2d_pair(smem + P::kQ + x * P::kQTile + half * (kBlockM * 128), &tm_q, q_full0, half * 64,
+                                     q_row + x * 2 * kBlockM);
+            const int sel_base = sel_identity ? (b * Hkv + kvh) * N : bh * sel_rows;
+            bool ok = true;
+            int armed_k = 0, armed_v = 0, spins = 0;
+            long long t0 = clock64();
+            while (armed_k < st.n_tiles || armed_v < st.n_tiles) {
+                bool progressed = false;
+                if (armed_k < st.n_tiles) {
+                    const int i = armed_k, ks = i % P::kKStages;
+                    if (mbar_try_wait(k_empty + ks, ((i / P::kKStages) & 1) ^ 1)) {
+                        const bool sel = st.is_sel(i);
+                        const int row = (sel ? sel_base + i * kBlockN : (b * Hkv + kvh) * N + st.loc_m(i) * kBlockN) +
+                                        (int)rank * (kBlockN / 2);   // this CTA's 64 keys
+                        if (rank == 0) mbar_expect_tx(k_full + ks, 2 * P::kKHalf);
+                        for (int half = 0; half < D / 64; ++half)
+                            tma_load_2d_pair(smem + P::kK + ks * P::kKHalf + half * ((kBlockN / 2) * 128), sel ? &tm_ksel : &tm_k,
+                                             k_full0 + ks * 8, half * 64, row);
+                        ++armed_k;
+                        progressed = true;
+                    }
+                }
+                if (armed_v < st.n_tiles) {
+                    const int i = armed_v, vs = i % P::kVStages;
+                    if (mbar_try_wait(v_empty + vs, ((i / P::kVStages) & 1) ^ 1)) {
+                        const bool sel = st.is_sel(i);
+                        const int row = sel ? sel_base + i * kBlockN : (b * Hkv + kvh) * N + st.loc_m(i) * kBlockN;
+                        if (rank == 0) mbar_expect_tx(v_full + vs, 2 * P::kVHalf);
+                        for (int q = 0; q < D / 128; ++q)           // this CTA's D / 2 value columns, 64 at a time
+                            tma_load_2d_pair(smem + P::kV + vs * P::kVHalf + q * (kBlockN * 128), sel ? &tm_vsel : &tm_v,
+                                             v_full0 + vs * 8, (int)rank * (D / 2) + q * 64, row);
+                        ++armed_v;
+                        progressed = true;
+                    }
+                }
+                if (progressed) {
+                    spins = 0;
+                } else if ((++spins & 1023) == 0) {
+                    if (spins == 1024) t0 = clock64();
+                    if (*abort_flag) { ok = false; break; }
+                    if (clock64() - t0 > kWaitLimitCycles) {
+                        *abort_flag = 1;
+                        report_status(status, STILL_ERR_DEVICE_TIMEOUT, 51);
+                        ok = false;
+                        break;
+                    }
+                }
+            }
+            if (!ok) {
+                tell_peer();
+                // leave no copy in flight behind: rank 0 waits (bounded) for the last stages armed, which count
+                // both CTAs' bytes; rank 1, whose copies complete on rank 0's barriers, waits out a fixed
+                // stretch that is long against a tile load
+                if (rank == 0) {
+                    if (armed_k > 0) mbar_wait_drain(k_full + (armed_k - 1) % P::kKStages, ((armed_k - 1) / P::kKStages) & 1);
+                    if (armed_v > 0) mbar_wait_drain(v_full + (armed_v - 1) % P::kVStages, ((armed_v - 1) / P::kVStages) & 1);
+                } else {
+                    const long long t1 = clock64();
+                    while (clock64() - t1 < 200000) {}
+                }
+            }
+        }
+    } else if (warp == 1 && rank == 0) {
+        // ------------------------------------------------------------ MMA issuer (rank 0 only)
+        if (lane == 0) {
+            constexpr uint32_t idesc_qk = make_idesc(2 * kBlockM, kBlockN, false);
+            constexpr uint32_t idesc_pv = make_idesc(2 * kBlockM, D, true);
+            bool ok = mbar_wait(q_full, 0, abort_flag, status, 54);
+            tc_fence_after();
+            const uint32_t q_lo0 = desc_lo(smem_u32(smem + P::kQ), 0);
+            const uint32_t k_lo0 = desc_lo(smem_u32(smem + P::kK), 0);
+            const uint32_t v_lo0 = desc_lo(smem_u32(smem + P::kV), kBlockN * 128);
+            const uint32_t k_empty1 = mapa(smem_u32(k_empty), 1), v_empty1 = mapa(smem_u32(v_empty), 1);
+            int pending[2] = {-1, -1};
+            int n_done[2] = {0, 0};
+            auto issue_pv = [&](int x, int ip) -> bool {
+                const int vs = ip % P::kVStages;
+                if (!mbar_wait(v_full + vs, (ip / P::kVStages) & 1, abort_flag, status, 56)) return false;
+                if (!mbar_wait(p_half + 2 * x, n_done[x] & 1, abort_flag, status, 55)) return false;
+                tc_fence_after();
+                const uint32_t v_lo = v_lo0 + vs * (P::kVHalf >> 4);
+                const uint32_t d_o = tmem_base + col_o(x), a_p = tmem_base + col_s(x);
+#pragma unroll
+                for (int k = 0; k < kBlockN / 32; ++k)
+                    mma_ts_lo_pair<idesc_pv>(d_o, a_p + k * 8, v_lo + k * (16 * 128 >> 4), (n_done[x] > 0 || k > 0) ? 1u : 0u);
+                if (!mbar_wait(p_half + 2 * x + 1, n_done[x] & 1, abort_flag, status, 55)) return false;
+                tc_fence_after();
+#pragma unroll
+                for (int k = kBlockN / 32; k < kBlockN / 16; ++k)
+                    mma_ts_lo_pair<idesc_pv>(d_o, a_p + k * 8, v_lo + k * (16 * 128 >> 4), 1u);
+                ++n_done[x];
+                return true;
+            };
+            for (int i = 0; i < st.n_tiles && ok; ++i) {
+                const int ks = i % P::kKStages;
+                ok = mbar_wait(k_full + ks, (i / P::kKStages) & 1, abort_flag, status, 57);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t k_lo = k_lo0 + ks * (P::kKHalf >> 4);
+                for (int x = 0; x < 2 && ok; ++x) {
+                    const bool present = (x == 0) || st.has_b;
+                    if (present && st.used_by(x, i)) {
+                        if (pending[x] >= 0) {
+                            const int ip = pending[x];
+                            ok = issue_pv(x, ip);
+                            if (!ok) break;
+                            // a V stage is released by two arrivals per CTA: pay the other tile's share if it skipped ip
+                            if (!(((1 - x) == 0 || st.has_b) && st.used_by(1 - x, ip))) {
+                                mbar_arrive(v_empty + ip % P::kVStages);
+                                mbar_arrive_cluster(v_empty1 + (ip % P::kVStages) * 8);
+                            }
+                        }
+                        const uint32_t q_lo = q_lo0 + x * (P::kQTile >> 4), d_s = tmem_base + col_s(x);
+                        mma_ss_lo_pair<idesc_qk, 0>(d_s, q_lo, k_lo);
+#pragma unroll
+                        for (int k = 1; k < D / 16; ++k) {
+                            // k-step of 16 elements: 32 bytes within a 64-element swizzle atom; atoms are 128 rows
+                            // apart in a Q tile, 64 rows apart in a CTA's half of a K tile
+                            const uint32_t off_q = ((k / 4) * (kBlockM * 128) + (k % 4) * 32) >> 4;
+                            const uint32_t off_k = ((k / 4) * ((kBlockN / 2) * 128) + (k % 4) * 32) >> 4;
+                            mma_ss_lo_pair<idesc_qk, 1>(d_s, q_lo + off_q, k_lo + off_k);
+                        }
+                        tc_commit_pair(s_full + x, 3);
+                        pending[x] = i;
+                    } else {
+                        mbar_arrive(k_empty + ks);  // the share of a tile that skips this stream tile, in both CTAs
+                        mbar_arrive_cluster(k_empty1 + ks * 8);
+                    }
+                }
+            }
+            for (int x = 0; x < 2 && ok; ++x) {
+                if (pending[x] >= 0) {
+                    const int ip = pending[x];
+                    ok = issue_pv(x, ip);
+                    if (!ok) break;
+                    tc_commit_pair(o_final + x, 3);
+                }
+            }
+            if (!ok) {  // no MMA may still be running when tensor memory is freed
+                tell_peer();
+                tc_commit_pair_local(drain);
+                mbar_wait_drain(drain, 0);
+            }
+        }
+    }
+    } else {
+        reg_inc<216>();
+        // ------------------------------------------------------------ softmax + epilogue (both CTAs)
+        const int x = (warp - 4) >> 2;                 // 0: tile A, 1: tile B
+        softmax_role<D, P::kKStages, P::kVStages, true>(st, x, R0 + x * 2 * kBlockM + (int)rank * kBlockM, tmem_base, s_full,
+                                                        k_empty, v_empty, p_half, mapa(smem_u32(p_half), 0), o_final,
+                                                        abort_flag, status, smem + P::kQ + x * P::kQTile, N_LA, D_LA, Y, bh, N,
+                                                        C, lam, scale_log2);
+        if (*abort_flag) tell_peer();
+    }
+    // Nobody touches the peer's shared memory or tensor memory after this point.
+    tc_fence_before();
+    cluster_sync_all();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc_pair(tmem_base, 512);
     }
 }
 
@@ -868,22 +1191,35 @@ int launch_tc(const still_params_t *p, long long N, const void *Q, const void *K
         ++*launches;
         if (cudaGetLastError() != cudaSuccess) return STILL_ERR_CUDA;
     }
+    const unsigned long long kv_rows = (unsigned long long)p->B * p->Hkv * N;
+    const unsigned long long sel_total = identity ? kv_rows : (unsigned long long)BH * sel_rows;
+    constexpr bool kPair = D == 128;   // head dim 128 runs on CTA pairs, each CTA holding 64 keys of a K tile
     CUtensorMap tq, tk, tv, tks, tvs;
     if (!make_map(&tq, Q, (unsigned long long)BH * N, D) ||
-        !make_map(&tk, K, (unsigned long long)p->B * p->Hkv * N, D) ||
-        !make_map(&tv, V, (unsigned long long)p->B * p->Hkv * N, D) ||
-        !make_map(&tks, identity ? K : k_sel, identity ? (unsigned long long)p->B * p->Hkv * N : (unsigned long long)BH * sel_rows, D) ||
-        !make_map(&tvs, identity ? V : v_sel, identity ? (unsigned long long)p->B * p->Hkv * N : (unsigned long long)BH * sel_rows, D))
+        !make_map_2d(&tk, K, kv_rows, D, kPair ? kBlockN / 2 : kBlockN, false) || !make_map(&tv, V, kv_rows, D) ||
+        !make_map_2d(&tks, identity ? K : k_sel, sel_total, D, kPair ? kBlockN / 2 : kBlockN, false) ||
+        !make_map(&tvs, identity ? V : v_sel, sel_total, D))
         return STILL_ERR_CUDA;
-    const int n_qblocks = (int)((N + 2 * kBlockM - 1) / (2 * kBlockM));
-    if (ensure_dynamic_smem((const void *)sa_merge_tc_kernel<D>, SmemPlan<D>::kAlloc) != cudaSuccess)
-        return STILL_ERR_CUDA;
-    dim3 grid((unsigned)n_qblocks, (unsigned)BH);
-    profile_mark_begin(st);
-    sa_merge_tc_kernel<D><<<grid, kThreads, SmemPlan<D>::kAlloc, st>>>(
-        tq, tk, tv, tks, tvs, N_LA, D_LA, (bf *)Y, status, p->H, p->Hkv, (int)N, p->chunk, p->topk, (int)sel_rows, identity ? 1 : 0,
-        p->sm_scale * 1.4426950408889634f, n_qblocks);
-    profile_mark_end(st);
+    const float scale_log2 = p->sm_scale * 1.4426950408889634f;
+    if constexpr (kPair) {
+        const int n_pairs = (int)((N + 4 * kBlockM - 1) / (4 * kBlockM));
+        if (ensure_dynamic_smem((const void *)sa_merge_pair_kernel<D>, PairPlan<D>::kAlloc) != cudaSuccess) return STILL_ERR_CUDA;
+        dim3 grid((unsigned)(2 * n_pairs), (unsigned)BH);   // clusters of two along x
+        profile_mark_begin(st);
+        sa_merge_pair_kernel<D><<<grid, kThreads, PairPlan<D>::kAlloc, st>>>(
+            tq, tk, tv, tks, tvs, N_LA, D_LA, (bf *)Y, status, p->H, p->Hkv, (int)N, p->chunk, p->topk, (int)sel_rows,
+            identity ? 1 : 0, scale_log2, n_pairs);
+        profile_mark_end(st);
+    } else {
+        const int n_qblocks = (int)((N + 2 * kBlockM - 1) / (2 * kBlockM));
+        if (ensure_dynamic_smem((const void *)sa_merge_tc_kernel<D>, SmemPlan<D>::kAlloc) != cudaSuccess) return STILL_ERR_CUDA;
+        dim3 grid((unsigned)n_qblocks, (unsigned)BH);
+        profile_mark_begin(st);
+        sa_merge_tc_kernel<D><<<grid, kThreads, SmemPlan<D>::kAlloc, st>>>(
+            tq, tk, tv, tks, tvs, N_LA, D_LA, (bf *)Y, status, p->H, p->Hkv, (int)N, p->chunk, p->topk, (int)sel_rows,
+            identity ? 1 : 0, scale_log2, n_qblocks);
+        profile_mark_end(st);
+    }
     ++*launches;
     if (cudaGetLastError() != cudaSuccess) return STILL_ERR_CUDA;
     return STILL_OK;
