@@ -52,7 +52,7 @@ static inline bool la_active(const still_params_t *p) { return p->topk < p->chun
 
 // Workspace plan of the prefill.
 struct FwdPlan {
-    size_t status, scores, sel_idx, phiQ, phiK, nla, dla, ksel, vsel, total;
+    size_t status, scores, sel_idx, phiQ, phiK, csum, zpre, nla, dla, ypart, dpart, ksel, vsel, total;
     long long T, sel_rows;  // chunks; rows of the compacted salient K/V per head
     bool la, tc, tc_la;
 };
@@ -76,10 +76,21 @@ static FwdPlan plan_fwd(const still_params_t *p, long long N) {
     w.scores = take(BH * (size_t)N * 4);
     w.sel_idx = take(BH * (size_t)T * (size_t)std::max(p->topk, 1) * 4);
     if (w.la) {
-        w.phiQ = take(BH * (size_t)N * dp * (w.tc_la ? 4 : es));  // fp32 features for the TF32 read-out GEMM
         w.phiK = take(BHkv * (size_t)N * dp * es);
-        w.nla = take(BH * (size_t)N * p->d * 4);
-        w.dla = take(BH * (size_t)N * 4);
+        if (w.tc_la) {
+            // tensor-core branch: phi(Q) is never stored; the branch leaves two bf16 partial results
+            w.csum = take(BHkv * (size_t)T * dp * 4);
+            w.zpre = take(BH * (size_t)std::max<long long>(T - 2, 1) * dp * 4);
+        } else {
+            w.phiQ = take(BH * (size_t)N * dp * es);
+            w.nla = take(BH * (size_t)N * p->d * 4);
+            w.dla = take(BH * (size_t)N * 4);
+        }
+        if (w.tc) {
+            const int parts = w.tc_la ? 2 : 1;
+            w.ypart = take(parts * BH * (size_t)N * p->d * 2);
+            w.dpart = take(parts * BH * (size_t)N * 4);
+        }
     }
     if (w.tc) {
         w.sel_rows = tc_sel_rows(p, N);
@@ -272,22 +283,36 @@ static int fwd_typed(const still_params_t *p, long long N, const T *Q, const T *
     if (rc != STILL_OK) return rc;
 
     // (3) NP-Map + linear-attention scan (skipped when no token can be in M^LA).
-    float *nla = nullptr, *dla = nullptr;
+    float *nla = nullptr, *dla = nullptr, *dpart = nullptr;
+    void *ypart = nullptr;
+    int n_parts = 0;
     float *S_out = state ? reinterpret_cast<float *>(state + L.S) : nullptr;
     float *z_out = state ? reinterpret_cast<float *>(state + L.z) : nullptr;
     if (w.la) {
-        T *phiQ = reinterpret_cast<T *>(ws + w.phiQ), *phiK = reinterpret_cast<T *>(ws + w.phiK);
-        nla = reinterpret_cast<float *>(ws + w.nla);
-        dla = reinterpret_cast<float *>(ws + w.dla);
+        T *phiK = reinterpret_cast<T *>(ws + w.phiK);
         if (w.tc_la) {
-            rc = tc_la_branch(p, N, Q, K, V, G, Wq, bq, Wk, bk, sel, phiQ, phiK, nla, dla, S_out, z_out,
+            ypart = ws + w.ypart;
+            dpart = reinterpret_cast<float *>(ws + w.dpart);
+            n_parts = 2;
+            rc = tc_la_branch(p, N, Q, K, V, G, Wq, bq, Wk, bk, sel, phiK, reinterpret_cast<float *>(ws + w.csum),
+                              reinterpret_cast<float *>(ws + w.zpre), ypart, dpart, S_out, z_out,
                               reinterpret_cast<int *>(ws + w.status), st, &g_launches);
             if (rc != STILL_OK) return rc;
         } else {
+            T *phiQ = reinterpret_cast<T *>(ws + w.phiQ);
+            nla = reinterpret_cast<float *>(ws + w.nla);
+            dla = reinterpret_cast<float *>(ws + w.dla);
             if ((rc = launch_npmap<T>(p, N, p->H, Q, Wq, bq, phiQ, st)) != STILL_OK) return rc;
             if ((rc = launch_npmap<T>(p, N, p->Hkv, K, Wk, bk, phiK, st)) != STILL_OK) return rc;
             if ((rc = launch_la_scan<T>(p, N, w.T, phiQ, phiK, V, G, sel, nla, dla, S_out, z_out, st)) != STILL_OK)
                 return rc;
+            if (w.tc && Y) {   // the tensor-core attention kernel takes the linear branch as bf16 parts
+                ypart = ws + w.ypart;
+                dpart = reinterpret_cast<float *>(ws + w.dpart);
+                n_parts = 1;
+                if ((rc = tc_la_to_part(nla, dla, ypart, dpart, (long long)p->B * p->H * N, p->d, st, &g_launches)) != STILL_OK)
+                    return rc;
+            }
         }
     } else if (state) {
         STILL_CUDA(cudaMemsetAsync(state + L.S, 0, L.scratch - L.S, st));
@@ -296,7 +321,7 @@ static int fwd_typed(const still_params_t *p, long long N, const T *Q, const T *
     // (4) softmax-attention branch + merge.
     if (Y) {
         if (w.tc) {
-            rc = tc_sa_merge(p, N, Q, K, V, sel, nla, dla, Y, ws + w.ksel, ws + w.vsel, w.sel_rows,
+            rc = tc_sa_merge(p, N, Q, K, V, sel, ypart, dpart, n_parts, Y, ws + w.ksel, ws + w.vsel, w.sel_rows,
                              reinterpret_cast<int *>(ws + w.status), st, &g_launches);
         } else {
             profile_mark_begin(st);

@@ -1,32 +1,37 @@
 // Linear-attention branch of the prefill on tensor cores (bf16 inputs, sm_100a).
 //
-// Two kernels:
+// npmap_tc_kernel -- Norm-Preserved Feature Map (Sec. 3.2, Eq. feature_map) of 128 rows of K per CTA,
+//   fused into the load of the rows:  f = x W  on tcgen05 (x tile K-major from TMA, W MN-major from TMA,
+//   accumulator in TMEM), then per row  u = (f + b) ||x|| / max(||f + b||, 1e-12),
+//   phi = [softmax(u), softmax(-u)], stored as bf16 (the B operand of the bf16 state-update GEMM) once
+//   per KV head, together with the column sums of every chunk.
 //
-// npmap_tc_kernel -- Norm-Preserved Feature Map (Sec. 3.2, Eq. feature_map) of 128 rows of Q or K
-//   per CTA, fused into the load of the rows:  f = x W  on tcgen05 (x tile K-major from TMA, W
-//   MN-major from TMA, accumulator in TMEM), then per row  u = (f + b) ||x|| / max(||f + b||, 1e-12),
-//   phi = [softmax(u), softmax(-u)].  phi(K) is stored as bf16 (it is the B operand of the bf16
-//   state-update GEMM), phi(Q) as fp32 (B operand of the TF32 read-out GEMM).
+// z_delta_kernel / z_scan_kernel -- the normaliser z of Eq. cache_routing_sum after every routed chunk:
+//   column sums of the chunk minus the rows of its selected tokens, then a running sum over chunks.
 //
-// la_scan_tc_kernel -- Algorithm 1 "Linear Attention Branch" with the state of Eq.
-//   cache_routing_sum kept in tensor memory.  One CTA owns one (batch, query head) and 64 of the d
-//   value columns and walks the chunks in order.  The state is held transposed, S^T [128 x d']
-//   fp32 in TMEM: lanes 0-63 are the 64 value columns, lane 64 is the normaliser z (the A operand
-//   of the update has a second 64-row atom whose first row is all ones), lanes 65-127 are zero.
-//     update   S^T += [V_c^T ; 1] phi_k(K_c)   for the chunk c that has just left the two-chunk
-//              local region: bf16 UMMA, A = V tile (M-major, as TMA delivers it), B = phi(K) tile
-//              (MN-major) whose rows of the tokens selected for softmax attention were zeroed;
-//     read-out [N_LA^T ; D_LA] = S^T phi_q(Q_c)^T  for the chunk c being answered: TF32 UMMA with
-//              the fp32 state read straight from TMEM as the A operand (no conversion pass; 10-bit
-//              mantissa instead of the 7 bits a bf16 copy of the state would keep), B = phi(Q)
-//              tile (K-major fp32).
-//   The lag of two chunks between update and read-out is the delayed selection of Sec. 3.3.
-//   Work is tiled in 64-token sub-chunks, so C = 128 is two sub-chunks per chunk.
+// la_fused_kernel -- Algorithm 1 "Linear Attention Branch" with the state of Eq. cache_routing_sum kept
+//   in tensor memory and the query-side NP-Map computed on the fly (phi(Q) never reaches HBM).  One CTA
+//   owns one (batch, query head) and one half of the feature dimension (the softmax(u) features or the
+//   softmax(-u) features) and walks the chunks in order.  The state half is held transposed, S^T
+//   [value columns x d_f features] fp32 in TMEM.
+//     update   S^T += V_c^T phi_k(K_c)   for the chunk c that has just left the two-chunk local region:
+//              bf16 UMMA, A = V tile (M-major, as TMA delivers it), B = phi(K) half tile (MN-major)
+//              whose rows of the tokens selected for softmax attention were zeroed;
+//     map      f = Q W_q for a block of 128 query rows (UMMA), then a thread per row: norm re-injection,
+//              this CTA's softmax half, written unnormalised (e_j = 2^(+-u_j - max)) as an fp32 K-major
+//              tile into shared memory; D_part = (e . z_half of the chunk two back) / sum e;
+//     read-out N_part^T = S^T phi_q(Q_c)^T  for the chunk c being answered: TF32 UMMA with the fp32
+//              state read straight from TMEM as the A operand (10-bit mantissa instead of the 7 bits a
+//              bf16 copy of the state would keep), B = the phi(Q) tile.
+//   Output: y_part = N_part / D_part = (e . S) / (e . z) (times the gate) as bf16 and D_part as fp32, per feature half; the
+//   merge epilogue of the attention kernel forms N_LA = sum y_part D_part, D_LA = sum D_part.
+//   The lag of two chunks between update and read-out is the delayed selection of Sec. 3.3.  Work is
+//   tiled in 64-token sub-chunks, so C = 128 is two sub-chunks per chunk.
 //
-// Roles (192 threads): warp 0 TMA producer, warp 1 MMA issuer, warps 2-5 zero the selected rows of
-// the phi(K) tiles and run the epilogue (N_LA times the gate, D_LA, final state).  Every mbarrier
-// wait is bounded; on expiry the kernel records STILL_ERR_DEVICE_TIMEOUT in the status word, all
-// roles leave their loops and tensor memory is freed before the CTA exits.
+// Roles of la_fused_kernel (384 threads): warp 0 TMA producer, warp 1 MMA issuer, warp 2 zeroes the
+// selected rows of the phi(K) tiles, warps 4-7 write the output, warps 8-11 the query-side map.  Every mbarrier
+// wait is bounded; on expiry the kernel records STILL_ERR_DEVICE_TIMEOUT in the status word, all roles
+// leave their loops and tensor memory is freed before the CTA exits.
 #include "still_tc.h"
 
 #include <algorithm>
@@ -71,7 +76,8 @@ struct NpmapSmem {
 template <int D, int DF, typename TOut>
 __global__ void __launch_bounds__(192, 3)
 npmap_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
-                const __nv_bfloat16 *__restrict__ bias, TOut *__restrict__ phi, int *status, int heads, int N) {
+                const __nv_bfloat16 *__restrict__ bias, TOut *__restrict__ phi, float *__restrict__ csum, int *status,
+                int heads, int N, int C) {
     constexpr int kXBytes = 128 * D * 2, kWBytes = D * DF * 2;
     using Lay = NpmapSmem<D, DF, TOut>;
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -191,6 +197,7 @@ npmap_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
             constexpr int kHalfChunks = Lay::kHalfChunks, kStageRow = Lay::kStageRow;
             uint8_t *stage = smem + wq * (32 * kStageRow);
             const int rows_live = min(32, N - (R0 + wq * 32));        // rows of this warp that exist
+            float *csw = reinterpret_cast<float *>(smem + 4 * 32 * kStageRow) + wq * (2 * DF);   // this warp's column sums
 #pragma unroll 1
             for (int q = 0; q < DF / 32; ++q) {
                 uint32_t v[32];
@@ -221,6 +228,20 @@ npmap_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
                     }
                 }
                 __syncwarp();
+                if constexpr (sizeof(TOut) == 2) {
+                    // column sums of the stored (bf16-rounded) features over the warp's rows, in row order: lane l
+                    // adds feature 32 q + l of both halves (what the normaliser z of the linear branch is made of)
+                    if (csum != nullptr) {
+                        float sp = 0.f, sn = 0.f;
+                        for (int row = 0; row < rows_live; ++row) {
+                            const uint8_t *src = stage + row * kStageRow + lane * 2;
+                            sp += __uint_as_float((uint32_t)(*reinterpret_cast<const uint16_t *>(src)) << 16);
+                            sn += __uint_as_float((uint32_t)(*reinterpret_cast<const uint16_t *>(src + kHalfChunks * 16)) << 16);
+                        }
+                        csw[q * 32 + lane] = sp;
+                        csw[DF + q * 32 + lane] = sn;
+                    }
+                }
 #pragma unroll
                 for (int it = 0; it < 2 * kHalfChunks; ++it) {
                     const int id = it * 32 + lane, row = id / (2 * kHalfChunks), c = id % (2 * kHalfChunks);
@@ -238,6 +259,22 @@ npmap_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
     }
     tc_fence_before();
     __syncthreads();
+    if constexpr (sizeof(TOut) == 2) {
+        // per-chunk column sums: the warps of a chunk are added in warp order (fixed order: the sums are reproducible)
+        if (csum != nullptr && warp >= 2 && !*abort_flag) {
+            const float *csw_all = reinterpret_cast<const float *>(smem + 4 * 32 * NpmapSmem<D, DF, TOut>::kStageRow);
+            const int Tn = (N + C - 1) / C, wpc = C / 32;             // warps (of 32 rows) per chunk: 2 or 4
+            for (int i = threadIdx.x - 64; i < (128 / C) * 2 * DF; i += 128) {
+                const int k = i / (2 * DF), f = i % (2 * DF), chunk = R0 / C + k;
+                if (chunk < Tn) {
+                    float acc = 0.f;
+                    for (int w = 0; w < wpc; ++w)
+                        if (R0 + (k * wpc + w) * 32 < N) acc += csw_all[(k * wpc + w) * (2 * DF) + f];
+                    csum[(((long long)b * heads + hd) * Tn + chunk) * (2 * DF) + f] = acc;
+                }
+            }
+        }
+    }
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, 128);
@@ -245,48 +282,101 @@ npmap_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
 }
 
 // ------------------------------------------------------------------------------------------
-// State scan
+// Normaliser prefix z (Eq. cache_routing_sum): z after chunk c = sum over the chunks 0..c of the features
+// of their unselected tokens = (column sums of phi(K) over the chunk) - (rows of its selected tokens).
 // ------------------------------------------------------------------------------------------
-template <int NF>  // feature dim d' = 2 d_f: 128 or 256
-struct ScanPlan {
-    static constexpr int kPhiK = 64 * NF * 2;          // phi(K) tile of 64 tokens, bf16
-    static constexpr int kVt = 64 * 64 * 2;            // V tile: 64 tokens x 64 value columns, bf16
-    static constexpr int kUStage = kPhiK + kVt;
-    static constexpr int kPhiQ = 64 * NF * 4;          // phi(Q) tile of 64 tokens, fp32
-    static constexpr int kU = 0;                       // two update stages
-    static constexpr int kQ = kU + 2 * kUStage;        // two read-out stages
-    static constexpr int kOnes = kQ + 2 * kPhiQ;       // second M atom of the update's A operand
-    static constexpr int kBar = kOnes + 64 * 128;
-    static constexpr int kNumBars = 2 + 2 + 2 + 2 + 2 + 5;  // u_full, u_empty, u_masked, q_full, q_empty, r_done[2], out_free[2], fin
-    static constexpr int kMisc = kBar + kNumBars * 8;
-    static constexpr int kTotal = kMisc + 16;
-};
-static_assert(ScanPlan<128>::kTotal <= 232448 && ScanPlan<256>::kTotal <= 232448,
-              "state scan: the shared-memory plan exceeds what a CTA can have");
+// grid (routed chunks, B*H), 2 d_f threads: zpre[bh][c][f] = csum[kv][c][f] - sum_i phi(K)[sel[bh][c][i]][f]
+__global__ void z_delta_kernel(const float *__restrict__ csum, const __nv_bfloat16 *__restrict__ phiK,
+                               const int32_t *__restrict__ sel_idx, float *__restrict__ zpre, int H, int Hkv, long long N,
+                               int Tn, int n_routed, int lam, int NF) {
+    const int c = blockIdx.x, bh = blockIdx.y, b = bh / H, h = bh % H, kv = b * Hkv + h / (H / Hkv), f = threadIdx.x;
+    float d = csum[((long long)kv * Tn + c) * NF + f];
+    const int32_t *si = sel_idx + ((long long)bh * Tn + c) * lam;
+    for (int i = 0; i < lam; ++i) {
+        const int p = si[i];
+        if (p >= 0) d -= __bfloat162float(phiK[((long long)kv * N + p) * NF + f]);
+    }
+    zpre[((long long)bh * n_routed + c) * NF + f] = d;
+}
+// grid (B*H), 2 d_f threads: in-place running sum over the routed chunks; the last value is the state's z.
+__global__ void z_scan_kernel(float *__restrict__ zpre, float *__restrict__ z_out, int n_routed, int NF) {
+    const int bh = blockIdx.x, f = threadIdx.x;
+    float *z = zpre + (long long)bh * n_routed * NF + f;
+    float acc = 0.f;
+    for (int c0 = 0; c0 < n_routed; c0 += 8) {   // eight independent loads in flight, then the running sum
+        float v[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[i] = c0 + i < n_routed ? z[(long long)(c0 + i) * NF] : 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            acc += v[i];
+            if (c0 + i < n_routed) z[(long long)(c0 + i) * NF] = acc;
+        }
+    }
+    if (z_out != nullptr) z_out[(long long)bh * NF + f] = acc;
+}
 
-template <int NF>
-__global__ void __launch_bounds__(192, 1)
-la_scan_tc_kernel(const __grid_constant__ CUtensorMap tm_phik, const __grid_constant__ CUtensorMap tm_v,
-                  const __grid_constant__ CUtensorMap tm_phiq, const __nv_bfloat16 *__restrict__ G,
-                  const int32_t *__restrict__ sel_idx, float *__restrict__ N_LA, float *__restrict__ D_LA,
-                  float *__restrict__ S_out, float *__restrict__ z_out, int *status, int H, int Hkv, int N, int d,
-                  int C, int lam) {
-    using P = ScanPlan<NF>;
+// ------------------------------------------------------------------------------------------
+// State scan with the query-side NP-Map fused into its loads
+// ------------------------------------------------------------------------------------------
+// One CTA owns one (batch, query head) and one half of the feature dimension: the softmax(u) half or the
+// softmax(-u) half of phi (each d_f features).  N_LA and D_LA are sums over features, so the two CTAs of a
+// head produce two partial results that the merge epilogue of the attention kernel adds.
+template <int D, int DF>
+struct FusedPlan {
+    static constexpr int kW = D * DF * 2;               // W_q, MN-major (as TMA delivers [d rows, d_f columns])
+    static constexpr int kX = 128 * D * 2;              // raw Q rows of one block of 128 tokens
+    static constexpr int kPhiQ = 64 * DF * 4;           // phi_q half of 64 tokens, fp32 (TF32 operand)
+    static constexpr int kPhiK = 64 * DF * 2;           // phi_k half of 64 tokens, bf16
+    static constexpr int kVt = 64 * D * 2;              // V of 64 tokens
+    static constexpr int kUStage = kPhiK + kVt;
+    static constexpr int oW = 0;
+    static constexpr int oX = oW + kW;
+    static constexpr int oQ = oX + kX;                  // two slots
+    static constexpr int oU = oQ + 2 * kPhiQ;           // two stages
+    static constexpr int oDinv = oU + 2 * kUStage;      // [8][64] 1 / D_part of the tokens of the last sub-chunks
+    static constexpr int oZ = oDinv + 8 * 64 * 4;       // [4 map warps][d_f] z half of the chunk two back
+    static constexpr int oStage = oZ + 4 * DF * 4;      // [64 tokens][d] bf16: the output of a sub-chunk on its way out
+    static constexpr int oBar = oStage + 64 * D * 2;
+    static constexpr int kNumBars = 24;
+    static constexpr int oMisc = oBar + kNumBars * 8;
+    static constexpr int kTotal = oMisc + 16;
+};
+static_assert(FusedPlan<128, 128>::kTotal <= 232448 && FusedPlan<128, 64>::kTotal <= 232448 && FusedPlan<64, 64>::kTotal <= 232448,
+              "fused scan: the shared-memory plan exceeds what a CTA can have");
+
+template <int D, int DF>
+__global__ void __launch_bounds__(384, 1)
+la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_wq,
+                const __grid_constant__ CUtensorMap tm_phik, const __grid_constant__ CUtensorMap tm_v,
+                const __nv_bfloat16 *__restrict__ bq, const __nv_bfloat16 *__restrict__ G,
+                const int32_t *__restrict__ sel_idx, const float *__restrict__ zpre, __nv_bfloat16 *__restrict__ y_part,
+                float *__restrict__ d_part, float *__restrict__ S_out, int *status, int H, int Hkv, int N, int C, int lam,
+                long long part_stride_y, long long part_stride_d) {
+    using P = FusedPlan<D, DF>;
+    constexpr int NF = 2 * DF;
     extern __shared__ __align__(1024) uint8_t smem[];
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + P::kBar);
-    uint64_t *u_full = bars, *u_empty = bars + 2, *u_masked = bars + 4, *q_full = bars + 6, *q_empty = bars + 8;
-    uint64_t *r_done = bars + 10, *out_free = bars + 12, *fin = bars + 14;
-    uint32_t *tmem_base_slot = reinterpret_cast<uint32_t *>(smem + P::kMisc);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + P::kMisc + 8);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + P::oBar);
+    uint64_t *w_full = bars, *x_full = bars + 1, *x_empty = bars + 2, *f_done = bars + 3, *f_free = bars + 4;
+    uint64_t *pq_full = bars + 5, *pq_empty = bars + 7, *u_full = bars + 9, *u_empty = bars + 11, *u_masked = bars + 13;
+    uint64_t *r_done = bars + 15, *out_free = bars + 17, *fin = bars + 19;
+    uint32_t *tmem_base_slot = reinterpret_cast<uint32_t *>(smem + P::oMisc);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + P::oMisc + 8);
+    float *dinv_ring = reinterpret_cast<float *>(smem + P::oDinv);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int bh = blockIdx.x, b = bh / H, h = bh % H, kvh = h / (H / Hkv);
-    const int e0 = blockIdx.y * 64;            // first value column of this CTA
+    const int half = blockIdx.y;                // 0: features softmax(u), 1: features softmax(-u)
     const int sc = C / 64;                      // 64-token sub-chunks per chunk
-    const int Tn = (N + C - 1) / C;             // chunks
+    const int Tn = (N + C - 1) / C;
     const int NU = (N + 63) / 64;               // sub-chunks with query rows
-    const int n_upd = Tn >= 3 ? (Tn - 2) * sc : 0;   // update tiles: sub-chunks of chunks 0 .. Tn-3
+    const int NB = (N + 127) / 128;             // blocks of 128 query rows
+    const int n_routed = Tn >= 3 ? Tn - 2 : 0;  // chunks whose tokens enter the state
+    const int n_upd = n_routed * sc;            // update tiles (sub-chunks of the routed chunks)
     const int u_first = 2 * sc;                 // first sub-chunk whose read-out sees a non-empty state
+    const int b_first = u_first / 2;            // its block
+    __nv_bfloat16 *y_out = y_part + (long long)half * part_stride_y;
+    float *d_out = d_part + (long long)half * part_stride_d;
 
     if ((smem_u32(smem) & 1023u) != 0) {
         if (threadIdx.x == 0) report_status(status, STILL_ERR_DEVICE_TIMEOUT, 97);
@@ -297,14 +387,17 @@ la_scan_tc_kernel(const __grid_constant__ CUtensorMap tm_phik, const __grid_cons
     if (*abort_flag) return;
     __syncthreads();
     if (threadIdx.x == 0) {
+        mbar_init(w_full, 1);
+        mbar_init(x_full, 1);
+        mbar_init(x_empty, 5);      // the f GEMM has read the rows (1) and so have the four map warps (4)
+        mbar_init(f_done, 1);
+        mbar_init(f_free, 4);
         for (int i = 0; i < 2; ++i) {
+            mbar_init(pq_full + i, 2);   // the two map warps that own the slot's 64 rows
+            mbar_init(pq_empty + i, 1);
             mbar_init(u_full + i, 1);
             mbar_init(u_empty + i, 1);
-            mbar_init(u_masked + i, 4);
-            mbar_init(q_full + i, 1);
-            mbar_init(q_empty + i, 4);
-        }
-        for (int i = 0; i < 2; ++i) {
+            mbar_init(u_masked + i, 1);
             mbar_init(r_done + i, 1);
             mbar_init(out_free + i, 4);
         }
@@ -312,16 +405,6 @@ la_scan_tc_kernel(const __grid_constant__ CUtensorMap tm_phik, const __grid_cons
         *abort_flag = 0;
         fence_barrier_init();
     }
-    // The "ones" atom: 64 token rows of 128 bytes; value column 0 (i.e. M index 64 of the A operand)
-    // is 1 for every token, everything else 0.  With the 128-byte swizzle, element 0 of row t sits in
-    // the 16-byte chunk (0 xor (t mod 8)).
-    for (int i = threadIdx.x; i < 64 * 128 / 4; i += blockDim.x) reinterpret_cast<uint32_t *>(smem + P::kOnes)[i] = 0u;
-    __syncthreads();
-    if (threadIdx.x < 64) {
-        const int t = threadIdx.x;
-        *reinterpret_cast<uint16_t *>(smem + P::kOnes + t * 128 + ((t & 7) << 4)) = 0x3f80;  // bf16 1.0
-    }
-    fence_proxy_async();
     if (warp == 1) {
         tmem_alloc(tmem_base_slot, 512);
         tmem_relinquish();
@@ -330,34 +413,42 @@ la_scan_tc_kernel(const __grid_constant__ CUtensorMap tm_phik, const __grid_cons
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_base_slot;
-    const uint32_t col_state = 0, col_out = NF;   // S^T [128 x NF] fp32; two read-out results [128 x 64] fp32, so that
-                                                  // the epilogue of one sub-chunk overlaps the MMAs of the next
+    // TMEM columns: S^T half [value lanes x d_f features] fp32; f = x W_q of a block [128 rows x d_f]; two read-out
+    // results [value lanes x 64 tokens]
+    constexpr uint32_t col_state = 0, col_f = DF, col_out = 2 * DF;
 
+    // Registers move from the first warpgroup (single-thread roles) to the map warps, whose threads hold a row of f
+    // (per scheduler: 72 + 152 + 224 registers for its three warps, of the 3 x 168 the CTA was launched with).
+    if (warp < 4) {
+    reg_dec<72>();
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
             const int kv_row0 = (b * Hkv + kvh) * N, q_row0 = bh * N;
-            int nu = 0, nq = 0;   // tiles requested so far
-            const int n_q = NU > u_first ? NU - u_first : 0;
-            int spins = 0;
+            const int n_blk = NB > b_first ? NB - b_first : 0;
+            if (n_blk > 0) {
+                mbar_expect_tx(w_full, P::kW);
+                for (int a = 0; a < DF / 64; ++a) tma_load_2d(smem + P::oW + a * (D * 128), &tm_wq, w_full, a * 64, h * D);
+            }
+            int nu = 0, nx = 0, spins = 0;
             long long t0 = clock64();
-            while (nu < n_upd || nq < n_q) {
+            while (nu < n_upd || nx < n_blk) {
                 bool progressed = false;
-                if (nu < n_upd && mbar_try_wait(u_empty + (nu & 1), ((nu >> 1) & 1) ^ 1)) {
-                    uint8_t *stg = smem + P::kU + (nu & 1) * P::kUStage;
-                    mbar_expect_tx(u_full + (nu & 1), P::kUStage);
-                    for (int a = 0; a < NF / 64; ++a)   // phi(K): MN-major, 64-feature atoms 64 rows apart
-                        tma_load_2d(stg + a * (64 * 128), &tm_phik, u_full + (nu & 1), a * 64, kv_row0 + nu * 64);
-                    tma_load_2d(stg + P::kPhiK, &tm_v, u_full + (nu & 1), e0, kv_row0 + nu * 64);
-                    ++nu;
+                if (nx < n_blk && mbar_try_wait(x_empty, (nx & 1) ^ 1)) {
+                    mbar_expect_tx(x_full, P::kX);
+                    for (int a = 0; a < D / 64; ++a)   // K-major, 64-element atoms 128 rows apart
+                        tma_load_2d(smem + P::oX + a * (128 * 128), &tm_q, x_full, a * 64, q_row0 + (b_first + nx) * 128);
+                    ++nx;
                     progressed = true;
                 }
-                if (nq < n_q && mbar_try_wait(q_empty + (nq & 1), ((nq >> 1) & 1) ^ 1)) {
-                    uint8_t *stg = smem + P::kQ + (nq & 1) * P::kPhiQ;
-                    mbar_expect_tx(q_full + (nq & 1), P::kPhiQ);
-                    for (int a = 0; a < NF / 32; ++a)   // phi(Q): K-major fp32, 32-feature atoms 64 rows apart
-                        tma_load_2d(stg + a * (64 * 128), &tm_phiq, q_full + (nq & 1), a * 32, q_row0 + (u_first + nq) * 64);
-                    ++nq;
+                if (nu < n_upd && mbar_try_wait(u_empty + (nu & 1), ((nu >> 1) & 1) ^ 1)) {
+                    uint8_t *stg = smem + P::oU + (nu & 1) * P::kUStage;
+                    mbar_expect_tx(u_full + (nu & 1), P::kUStage);
+                    for (int a = 0; a < DF / 64; ++a)  // phi(K) half: MN-major, 64-feature atoms 64 rows apart
+                        tma_load_2d(stg + a * (64 * 128), &tm_phik, u_full + (nu & 1), half * DF + a * 64, kv_row0 + nu * 64);
+                    for (int a = 0; a < D / 64; ++a)   // V: M-major A operand, 64-column atoms 64 rows apart
+                        tma_load_2d(stg + P::kPhiK + a * (64 * 128), &tm_v, u_full + (nu & 1), a * 64, kv_row0 + nu * 64);
+                    ++nu;
                     progressed = true;
                 }
                 if (progressed) {
@@ -367,178 +458,341 @@ la_scan_tc_kernel(const __grid_constant__ CUtensorMap tm_phik, const __grid_cons
                     if (*abort_flag) break;
                     if (clock64() - t0 > kWaitLimitCycles) {
                         *abort_flag = 1;
-                        report_status(status, STILL_ERR_DEVICE_TIMEOUT, 40);
+                        report_status(status, STILL_ERR_DEVICE_TIMEOUT, 60);
                         break;
                     }
                 }
             }
             if (*abort_flag) {  // leave no copy in flight behind
                 if (nu > 0) mbar_wait_drain(u_full + ((nu - 1) & 1), ((nu - 1) >> 1) & 1);
-                if (nq > 0) mbar_wait_drain(q_full + ((nq - 1) & 1), ((nq - 1) >> 1) & 1);
+                if (nx > 0) mbar_wait_drain(x_full, (nx - 1) & 1);
+                if (n_blk > 0) mbar_wait_drain(w_full, 0);
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            constexpr uint32_t idesc_upd = make_idesc(128, NF, true) | (1u << 15);  // A M-major, B MN-major
+            constexpr uint32_t idesc_f = make_idesc(128, DF, true);
+            constexpr uint32_t idesc_upd = make_idesc(128, DF, true) | (1u << 15);  // A M-major, B MN-major
             constexpr uint32_t idesc_rd = make_idesc_tf32(128, 64);
             bool ok = true;
-            int nu = 0, nq = 0;
+            int nu = 0, nq = 0, nx = 0;
+            // descriptors as low words: a k-step adds a constant (keeps this thread's instruction count low)
+            const uint32_t x_lo = desc_lo(smem_u32(smem + P::oX), 0), w_lo = desc_lo(smem_u32(smem + P::oW), D * 128);
+            const uint32_t q_lo0 = desc_lo(smem_u32(smem + P::oQ), 0);
+            const uint32_t pk_lo0 = desc_lo(smem_u32(smem + P::oU), 64 * 128);
+            const uint32_t v_lo0 = desc_lo(smem_u32(smem + P::oU + P::kPhiK), D == 128 ? 64 * 128 : 0);
+            // f = x W_q of block b_first + nx (the map warps have taken the previous f out of tensor memory)
+            auto issue_f = [&]() -> bool {
+                if (nx == 0 && !mbar_wait(w_full, 0, abort_flag, status, 61)) return false;
+                if (!mbar_wait(x_full, nx & 1, abort_flag, status, 62)) return false;
+                if (!mbar_wait(f_free, (nx & 1) ^ 1, abort_flag, status, 63)) return false;
+                tc_fence_after();
+#pragma unroll
+                for (int k = 0; k < D / 16; ++k) {
+                    const uint32_t xo = ((k / 4) * (128 * 128) + (k % 4) * 32) >> 4, wo = (k * (16 * 128)) >> 4;
+                    if (k == 0) mma_ss_lo<idesc_f, 0>(tmem_base + col_f, x_lo + xo, w_lo + wo);
+                    else mma_ss_lo<idesc_f, 1>(tmem_base + col_f, x_lo + xo, w_lo + wo);
+                }
+                tc_commit(f_done);
+                tc_commit(x_empty);
+                ++nx;
+                return true;
+            };
+            if (NB > b_first) ok = issue_f();
             for (int u = u_first; u < NU && ok; ++u) {
                 if (u % sc == 0) {
                     // the chunk that has just left the local region: sub-chunks of chunk u / sc - 2
                     for (int j = 0; j < sc && ok; ++j, ++nu) {
-                        ok = mbar_wait(u_masked + (nu & 1), (nu >> 1) & 1, abort_flag, status, 41);
+                        ok = mbar_wait(u_masked + (nu & 1), (nu >> 1) & 1, abort_flag, status, 64);
                         if (!ok) break;
                         tc_fence_after();
-                        const uint32_t stg = smem_u32(smem + P::kU + (nu & 1) * P::kUStage);
-                        const uint32_t v_addr = stg + P::kPhiK, ones = smem_u32(smem + P::kOnes);
+                        const uint32_t so = (uint32_t)(nu & 1) * (P::kUStage >> 4);
 #pragma unroll
                         for (int k = 0; k < 4; ++k)   // 16 tokens per step: 16 rows of 128 bytes in both operands
-                            mma_ss(tmem_base + col_state, smem_desc(v_addr + k * 2048, ones - v_addr),
-                                   smem_desc(stg + k * 2048, 64 * 128), idesc_upd, (nu > 0 || k > 0) ? 1u : 0u);
+                            mma_ss_lo_acc<idesc_upd>(tmem_base + col_state, v_lo0 + so + k * (2048 >> 4), pk_lo0 + so + k * (2048 >> 4),
+                                                     (nu > 0 || k > 0) ? 1u : 0u);
                         tc_commit(u_empty + (nu & 1));
                     }
                     if (!ok) break;
                 }
-                ok = mbar_wait(q_full + (nq & 1), (nq >> 1) & 1, abort_flag, status, 42);
-                if (ok) ok = mbar_wait(out_free + (nq & 1), ((nq >> 1) & 1) ^ 1, abort_flag, status, 43);
+                ok = mbar_wait(pq_full + (u & 1), (nq >> 1) & 1, abort_flag, status, 65);
+                if (ok) ok = mbar_wait(out_free + (nq & 1), ((nq >> 1) & 1) ^ 1, abort_flag, status, 66);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t qs = smem_u32(smem + P::kQ + (nq & 1) * P::kPhiQ);
+                const uint32_t q_lo = q_lo0 + (uint32_t)(u & 1) * (P::kPhiQ >> 4), d_out_t = tmem_base + col_out + (nq & 1) * 64;
 #pragma unroll
-                for (int k = 0; k < NF / 8; ++k)   // 8 features per step: 32 bytes within a 32-feature atom
-                    mma_ts_tf32(tmem_base + col_out + (nq & 1) * 64, tmem_base + col_state + k * 8,
-                                smem_desc(qs + (k / 4) * (64 * 128) + (k % 4) * 32, 0), idesc_rd, k > 0 ? 1u : 0u);
+                for (int k = 0; k < DF / 8; ++k) {   // 8 features per step: 32 bytes within a 32-feature atom
+                    const uint32_t qo = ((k / 4) * (64 * 128) + (k % 4) * 32) >> 4;
+                    if (k == 0) mma_ts_tf32_lo<idesc_rd, 0>(d_out_t, tmem_base + col_state, q_lo + qo);
+                    else mma_ts_tf32_lo<idesc_rd, 1>(d_out_t, tmem_base + col_state + k * 8, q_lo + qo);
+                }
                 tc_commit(r_done + (nq & 1));
+                tc_commit(pq_empty + (u & 1));
                 ++nq;
+                // the next block's f while this block's second sub-chunk is read out
+                if ((u & 1) == 0 && b_first + nx < NB) ok = issue_f();
             }
-            // state after the last update (chunks 0 .. Tn-3), for the decode state
-            if (ok) tc_commit(fin);
+            if (ok) tc_commit(fin);   // state after the last update, for the decode state
             if (!ok) {
                 tc_commit(fin);
                 mbar_wait_drain(fin, 0);
             }
         }
-    } else {
-        // ------------------------------------------------------------ workers: mask, epilogue
-        const int wq = warp & 3;                     // TMEM lane quarter this warp may read
-        const int e = wq * 32 + lane;                // lane of S^T / of the read-out result
-        const uint32_t taddr = tmem_base + ((uint32_t)(wq * 32) << 16);
-        const int tid = threadIdx.x - 64;            // 0..127
+    } else if (warp == 2) {
+        // ------------------------------------------------------------ mask warp
+        // Zeroes, in every phi(K) tile, the rows of the tokens kept for softmax attention: only the others enter the
+        // state.  The chunk's indices are fetched before the tile is waited for.
         bool ok = true;
-        int nu = 0, nq = 0;
-        // zero the rows of the tokens kept for softmax attention in update tile nu
-        auto mask_tile = [&]() {
-            if (ok) ok = mbar_wait(u_full + (nu & 1), (nu >> 1) & 1, abort_flag, status, 44);
+        for (int nu = 0; nu < n_upd; ++nu) {
+            const int chunk = nu / sc, sub = nu % sc;
+            const int32_t *si = sel_idx + ((long long)bh * Tn + chunk) * lam;
+            int row[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int i = lane + 32 * q;
+                row[q] = i < lam ? si[i] - (chunk * C + sub * 64) : -1;   // row within this 64-token tile
+            }
+            if (ok) ok = mbar_wait(u_full + (nu & 1), (nu >> 1) & 1, abort_flag, status, 67);
             ok = __all_sync(0xffffffffu, ok);
-            if (ok && lam > 0) {
-                const int chunk = nu / sc, sub = nu % sc;
-                const int32_t *si = sel_idx + ((long long)bh * Tn + chunk) * lam;
-                uint8_t *tile = smem + P::kU + (nu & 1) * P::kUStage;
-                // one token row = NF / 64 atoms x eight 16-byte pieces; a thread zeroes one piece at a time
-                constexpr int kPieces = NF / 8;
-                for (int i = tid; i < lam * kPieces; i += 128) {
-                    const int p = si[i / kPieces] - (chunk * C + sub * 64);   // row within this 64-token tile
-                    const int piece = i % kPieces;
-                    if (p >= 0 && p < 64)
-                        *reinterpret_cast<uint4 *>(tile + (piece >> 3) * (64 * 128) + p * 128 + ((piece & 7) << 4)) =
-                            make_uint4(0, 0, 0, 0);
-                }
+            if (ok) {
+                uint8_t *tile = smem + P::oU + (nu & 1) * P::kUStage;
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                    if (row[q] >= 0 && row[q] < 64) {
+#pragma unroll
+                        for (int piece = 0; piece < DF / 8; ++piece)   // 16-byte pieces of the token's feature half
+                            *reinterpret_cast<uint4 *>(tile + (piece >> 3) * (64 * 128) + row[q] * 128 + ((piece & 7) << 4)) =
+                                make_uint4(0, 0, 0, 0);
+                    }
                 fence_proxy_async();
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(u_masked + (nu & 1));
-            ++nu;
-        };
-        // rows of the first two chunks see an empty state
-        for (int i = tid; i < min(N, u_first * 64) * 64; i += 128) {
-            const int t = i >> 6, col = i & 63;
-            N_LA[((long long)bh * N + t) * d + e0 + col] = 0.f;
         }
-        if (blockIdx.y == 0)
-            for (int t = tid; t < min(N, u_first * 64); t += 128) D_LA[(long long)bh * N + t] = 0.f;
-
-        for (int j = 0; j < sc && nu < n_upd; ++j) mask_tile();       // tiles of the first update
+    }
+    } else if (warp < 8) {
+        reg_dec<152>();
+        // ------------------------------------------------------------ workers: output
+        const int wq = warp & 3;                     // TMEM lane quarter this warp may read
+        const int e = wq * 32 + lane;                // value column (lane of S^T and of the read-out result)
+        const uint32_t taddr = tmem_base + ((uint32_t)(wq * 32) << 16);
+        const int tid = threadIdx.x - 128;           // 0..127
+        bool ok = true;
+        int nq = 0;
+        // rows of the first two chunks see an empty state
+        {
+            const int n0 = min(N, u_first * 64);
+            for (int i = tid; i < n0 * (D / 8); i += 128)
+                reinterpret_cast<uint4 *>(y_out + (long long)bh * N * D)[i] = make_uint4(0, 0, 0, 0);
+            for (int t = tid; t < n0; t += 128) d_out[(long long)bh * N + t] = 0.f;
+        }
         for (int u = u_first; u < NU; ++u) {
-            if ((u + 1) % sc == 0)                                     // tiles of the next chunk's update
-                for (int j = 0; j < sc && nu < n_upd; ++j) mask_tile();
-            if (ok) ok = mbar_wait(r_done + (nq & 1), (nq >> 1) & 1, abort_flag, status, 45);
+            if (ok) ok = mbar_wait(r_done + (nq & 1), (nq >> 1) & 1, abort_flag, status, 68);
             ok = __all_sync(0xffffffffu, ok);
-            // The result leaves through shared memory (the phi(Q) stage this read-out has just consumed is free
-            // until the workers release it): a thread holds one value column of 64 tokens, but the rows of
-            // N_LA are token-major, and a column-wise store loop costs over a hundred clocks per instruction.
-            float *stg = reinterpret_cast<float *>(smem + P::kQ + (nq & 1) * P::kPhiQ);   // [64 tokens][64 columns], then D_LA [64]
-            const int base = u * 64;
             if (ok) {
                 tc_fence_after();
+                // the result is scaled by 1 / (e . z) of its token here (all loads of the scales come before the first
+                // store below: shared-memory loads are kept behind earlier stores)
+                const float4 *dinv = reinterpret_cast<const float4 *>(dinv_ring + (u & 7) * 64);
                 uint32_t o[64];
                 tmem_ld32(taddr + col_out + (nq & 1) * 64, o);
                 tmem_ld32(taddr + col_out + (nq & 1) * 64 + 32, o + 32);
                 tmem_wait_ld();
+#pragma unroll
+                for (int t4 = 0; t4 < 16; ++t4) {
+                    const float4 sc = dinv[t4];
+                    o[4 * t4] = __float_as_uint(__uint_as_float(o[4 * t4]) * sc.x);
+                    o[4 * t4 + 1] = __float_as_uint(__uint_as_float(o[4 * t4 + 1]) * sc.y);
+                    o[4 * t4 + 2] = __float_as_uint(__uint_as_float(o[4 * t4 + 2]) * sc.z);
+                    o[4 * t4 + 3] = __float_as_uint(__uint_as_float(o[4 * t4 + 3]) * sc.w);
+                }
                 tc_fence_before();
-                if (e < 64) {
+                __syncwarp();
+                if (lane == 0) mbar_arrive(out_free + (nq & 1));
+                // y_part[t][e] = N_part / D_part (times the gate).  A thread holds one value column of 64 tokens, but
+                // the rows of y_part are token-major and a store loop over tokens costs about a hundred clocks per
+                // instruction; so the tile is transposed through shared memory and leaves in 16-byte pieces.
+                __nv_bfloat16 *stg = reinterpret_cast<__nv_bfloat16 *>(smem + P::oStage);
+                if (e < D) {
 #pragma unroll
-                    for (int t = 0; t < 64; ++t) stg[t * 64 + e] = __uint_as_float(o[t]);
-                } else if (e == 64) {
-#pragma unroll
-                    for (int t = 0; t < 64; ++t) stg[64 * 64 + t] = __uint_as_float(o[t]);
+                    for (int t = 0; t < 64; ++t) stg[t * D + e] = __float2bfloat16_rn(__uint_as_float(o[t]));
                 }
             }
             asm volatile("bar.sync 2, 128;" ::: "memory");   // the four worker warps (always, whatever `ok`)
             if (ok) {
+                const int base = u * 64;
+                constexpr int kPiecesPerRow = D / 8;
 #pragma unroll
-                for (int it = 0; it < 8; ++it) {
-                    const int id = it * 128 + tid, t = id >> 4, c = id & 15;
+                for (int it = 0; it < 64 * kPiecesPerRow / 128; ++it) {
+                    const int id = it * 128 + tid, t = id / kPiecesPerRow, c = id % kPiecesPerRow;
                     if (base + t < N) {
-                        float4 v = *reinterpret_cast<const float4 *>(stg + t * 64 + c * 4);
-                        const long long off = ((long long)bh * N + base + t) * d + e0 + c * 4;
+                        uint4 v = *reinterpret_cast<const uint4 *>(smem + P::oStage + (t * D + c * 8) * 2);
+                        const long long off = ((long long)bh * N + base + t) * D + c * 8;
                         if (G != nullptr) {
-                            const uint2 gg = *reinterpret_cast<const uint2 *>(G + off);
-                            v.x *= __uint_as_float(gg.x << 16);
-                            v.y *= __uint_as_float(gg.x & 0xffff0000u);
-                            v.z *= __uint_as_float(gg.y << 16);
-                            v.w *= __uint_as_float(gg.y & 0xffff0000u);
+                            const uint4 gg = *reinterpret_cast<const uint4 *>(G + off);
+                            const uint32_t vw[4] = {v.x, v.y, v.z, v.w}, gw[4] = {gg.x, gg.y, gg.z, gg.w};
+                            uint32_t rw[4];
+#pragma unroll
+                            for (int q = 0; q < 4; ++q)
+                                rw[q] = pack_bf16(__uint_as_float(vw[q] << 16) * __uint_as_float(gw[q] << 16),
+                                                  __uint_as_float(vw[q] & 0xffff0000u) * __uint_as_float(gw[q] & 0xffff0000u));
+                            v = make_uint4(rw[0], rw[1], rw[2], rw[3]);
                         }
-                        *reinterpret_cast<float4 *>(N_LA + off) = v;
+                        *reinterpret_cast<uint4 *>(y_out + off) = v;
                     }
                 }
-                if (blockIdx.y == 0 && tid < 64 && base + tid < N) D_LA[(long long)bh * N + base + tid] = stg[64 * 64 + tid];
             }
-            asm volatile("bar.sync 2, 128;" ::: "memory");   // staging space read by all before the stage is released
-            if (lane == 0) {
-                mbar_arrive(out_free + (nq & 1));
-                mbar_arrive(q_empty + (nq & 1));
-            }
+            asm volatile("bar.sync 2, 128;" ::: "memory");   // the staging tile has been read before the next one is written
             ++nq;
         }
-        // final state for the decode state: S [d', d] and z [d']
+        // final state for the decode state: S [2 d_f, d], this CTA's features
         if (S_out != nullptr) {
             if (n_upd > 0) {
-                if (ok) ok = mbar_wait(fin, 0, abort_flag, status, 46);
+                if (ok) ok = mbar_wait(fin, 0, abort_flag, status, 69);
                 ok = __all_sync(0xffffffffu, ok);
                 if (ok) {
                     tc_fence_after();
 #pragma unroll 1
-                    for (int q = 0; q < NF / 32; ++q) {
+                    for (int q = 0; q < DF / 32; ++q) {
                         uint32_t sreg[32];
                         tmem_ld32(taddr + col_state + q * 32, sreg);
                         tmem_wait_ld();
-                        if (e < 64) {
+                        if (e < D) {
 #pragma unroll
                             for (int j = 0; j < 32; ++j)
-                                S_out[((long long)bh * NF + q * 32 + j) * d + e0 + e] = __uint_as_float(sreg[j]);
-                        } else if (e == 64 && blockIdx.y == 0) {
-#pragma unroll
-                            for (int j = 0; j < 32; ++j) z_out[(long long)bh * NF + q * 32 + j] = __uint_as_float(sreg[j]);
+                                S_out[((long long)bh * NF + half * DF + q * 32 + j) * D + e] = __uint_as_float(sreg[j]);
                         }
                     }
                 }
             } else {
-                for (int i = tid; i < NF * 64; i += 128) S_out[((long long)bh * NF + (i >> 6)) * d + e0 + (i & 63)] = 0.f;
-                if (blockIdx.y == 0)
-                    for (int i = tid; i < NF; i += 128) z_out[(long long)bh * NF + i] = 0.f;
+                for (int i = tid; i < DF * D; i += 128) S_out[((long long)bh * NF + half * DF) * D + i] = 0.f;
             }
+        }
+    } else {
+        reg_inc<224>();
+        // ------------------------------------------------------------ map warps: phi_q of a block of 128 rows
+        // A thread owns one row: u = (f + b) ||x|| / max(||f + b||, 1e-12); this CTA's half of phi is softmax(u) or
+        // softmax(-u) over all d_f features.  The row goes to the slot of its 64-token sub-chunk as fp32, K-major
+        // with the 128-byte swizzle the UMMA descriptor expects; D_part = phi_half . z_half of the chunk two back.
+        const int wq = warp & 3, r = wq * 32 + lane;   // TMEM lane quarter; row of the block
+        const uint32_t taddr = tmem_base + ((uint32_t)(wq * 32) << 16);
+        const __nv_bfloat16 *bias = bq != nullptr ? bq + (long long)h * DF : nullptr;
+        float *zs = reinterpret_cast<float *>(smem + P::oZ) + (warp - 8) * DF;   // this warp's copy of the z row
+        bool ok = true;
+        int nx = 0;
+        for (int blk = b_first; blk < NB; ++blk, ++nx) {
+            const int u = 2 * blk + (r >> 6);            // this row's sub-chunk; its slot is u & 1 = r >> 6
+            const int slot = r >> 6, rr = r & 63;
+            // z half of the chunk two back (every row of the warp dots its features with it): requested now,
+            // placed in shared memory when it is needed
+            float4 zreg = make_float4(0.f, 0.f, 0.f, 0.f);
+            {
+                const int chunk = min((u * 64) / C, Tn - 1);   // (a sub-chunk past the end of a ragged last block has no chunk)
+                const float *zrow = zpre + ((long long)bh * n_routed + (chunk - 2)) * NF + half * DF;
+                if (lane < DF / 4) zreg = reinterpret_cast<const float4 *>(zrow)[lane];
+            }
+            if (ok) ok = mbar_wait(x_full, nx & 1, abort_flag, status, 70);
+            ok = __all_sync(0xffffffffu, ok);
+            float nx2 = 0.f;
+            if (ok) {
+                float s4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int a = 0; a < D / 64; ++a)
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        const uint4 v = *reinterpret_cast<const uint4 *>(smem + P::oX + a * (128 * 128) + r * 128 + ((c ^ (r & 7)) << 4));
+                        const uint32_t w4[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const float lo = __uint_as_float(w4[q] << 16), hi = __uint_as_float(w4[q] & 0xffff0000u);
+                            s4[q] = fmaf(lo, lo, s4[q]);
+                            s4[q] = fmaf(hi, hi, s4[q]);
+                        }
+                    }
+                nx2 = (s4[0] + s4[1]) + (s4[2] + s4[3]);
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(x_empty);
+            if (lane < DF / 4) reinterpret_cast<float4 *>(zs)[lane] = zreg;
+            if (ok) ok = mbar_wait(f_done, nx & 1, abort_flag, status, 71);
+            ok = __all_sync(0xffffffffu, ok);
+            float fv[DF];
+            if (ok) {
+                tc_fence_after();
+#pragma unroll
+                for (int q = 0; q < DF / 32; ++q) tmem_ld32(taddr + col_f + q * 32, reinterpret_cast<uint32_t *>(fv) + q * 32);
+                tmem_wait_ld();
+                tc_fence_before();
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(f_free);
+            float sgn = 0.f, shift = 0.f;
+            if (ok) {
+                // (four independent chains each: the row is long and these are latency-bound reductions; this CTA's
+                // half needs only one extremum: max f for softmax(u), min f for softmax(-u))
+                float n2[4] = {0.f, 0.f, 0.f, 0.f}, ex[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+                const float unit = half == 0 ? 1.f : -1.f;
+#pragma unroll
+                for (int j = 0; j < DF; ++j) {
+                    if (bias != nullptr) fv[j] += __bfloat162float(bias[j]);
+                    n2[j & 3] = fmaf(fv[j], fv[j], n2[j & 3]);
+                    ex[j & 3] = fmaxf(ex[j & 3], fv[j] * unit);
+                }
+                const float nf2 = (n2[0] + n2[1]) + (n2[2] + n2[3]);
+                const float extreme = fmaxf(fmaxf(ex[0], ex[1]), fmaxf(ex[2], ex[3]));   // max of +-f
+                // u = f * ratio in the log2 domain; the exponent of this half is +-u - max(+-u) <= 0
+                const float ratio = sqrtf(nx2) / fmaxf(sqrtf(nf2), 1e-12f) * 1.4426950408889634f;
+                sgn = unit * ratio;
+                shift = -extreme * ratio;
+            }
+            // the slot is written only after the read-out that used it last has completed (every block fills both
+            // slots once)
+            if (ok) ok = mbar_wait(pq_empty + slot, (nx & 1) ^ 1, abort_flag, status, 72);
+            ok = __all_sync(0xffffffffu, ok);
+            if (ok) {
+                // The features go into the tile unnormalised, e_j = 2^(+-u_j - max): with D_part = (e . z) / sum e and
+                // N_part = (e . S) / sum e the output N_part / D_part = (e . S) / (e . z) does not need the sum, so the
+                // row is written as it is computed.  The z values of the next group of 16 features are loaded before
+                // the stores of this group (shared-memory loads are kept behind earlier stores).
+                uint8_t *tile = smem + P::oQ + slot * P::kPhiQ;
+                float zs4[4] = {0.f, 0.f, 0.f, 0.f}, ds4[4] = {0.f, 0.f, 0.f, 0.f};
+                float4 zc[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) zc[i] = *reinterpret_cast<const float4 *>(zs + 4 * i);
+#pragma unroll
+                for (int g = 0; g < DF / 16; ++g) {
+                    float4 zn[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i)
+                        zn[i] = g + 1 < DF / 16 ? *reinterpret_cast<const float4 *>(zs + 16 * (g + 1) + 4 * i) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int j = 16 * g + 4 * i;
+                        float4 ev;
+                        ev.x = ex2(fmaf(fv[j], sgn, shift));
+                        ev.y = ex2(fmaf(fv[j + 1], sgn, shift));
+                        ev.z = ex2(fmaf(fv[j + 2], sgn, shift));
+                        ev.w = ex2(fmaf(fv[j + 3], sgn, shift));
+                        zs4[0] += ev.x; zs4[1] += ev.y; zs4[2] += ev.z; zs4[3] += ev.w;
+                        ds4[0] = fmaf(ev.x, zc[i].x, ds4[0]);
+                        ds4[1] = fmaf(ev.y, zc[i].y, ds4[1]);
+                        ds4[2] = fmaf(ev.z, zc[i].z, ds4[2]);
+                        ds4[3] = fmaf(ev.w, zc[i].w, ds4[3]);
+                        // features j .. j+3: atom j / 32, 16-byte piece (j % 32) / 4, swizzled by the row
+                        *reinterpret_cast<float4 *>(tile + (j >> 5) * (64 * 128) + rr * 128 + ((((j & 31) >> 2) ^ (rr & 7)) << 4)) = ev;
+                    }
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) zc[i] = zn[i];
+                }
+                const float zsum = (zs4[0] + zs4[1]) + (zs4[2] + zs4[3]), draw = (ds4[0] + ds4[1]) + (ds4[2] + ds4[3]);
+                const int t = u * 64 + rr;
+                if (t < N) d_out[(long long)bh * N + t] = draw / zsum;     // D_part
+                dinv_ring[(u & 7) * 64 + rr] = draw > 0.f ? 1.f / draw : 0.f;
+                fence_proxy_async();
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(pq_full + slot);
         }
     }
     tc_fence_before();
@@ -552,48 +806,37 @@ la_scan_tc_kernel(const __grid_constant__ CUtensorMap tm_phik, const __grid_cons
 // ------------------------------------------------------------------------------------------ host side
 
 template <int D, int DF, typename TOut>
-int launch_npmap(const void *X, const void *W, const void *bias, void *phi, int B, int heads, long long N, int *status,
-                 cudaStream_t st, int *launches) {
+int launch_npmap(const void *X, const void *W, const void *bias, void *phi, float *csum, int B, int heads, long long N,
+                 int C, int *status, cudaStream_t st, int *launches) {
     CUtensorMap tx, tw;
     if (!make_map_2d(&tx, X, (unsigned long long)B * heads * N, D, 128, false) ||
         !make_map_2d(&tw, W, (unsigned long long)heads * D, DF, D, false))
         return STILL_ERR_CUDA;
     constexpr int kSmem = NpmapSmem<D, DF, TOut>::kTotal;
-    if (ensure_dynamic_smem((const void *)npmap_tc_kernel<D, DF, TOut>, kSmem) !=
-        cudaSuccess)
-        return STILL_ERR_CUDA;
+    if (ensure_dynamic_smem((const void *)npmap_tc_kernel<D, DF, TOut>, kSmem) != cudaSuccess) return STILL_ERR_CUDA;
     dim3 grid((unsigned)((N + 127) / 128), (unsigned)heads, (unsigned)B);
-    npmap_tc_kernel<D, DF, TOut><<<grid, 192, kSmem, st>>>(tx, tw, (const __nv_bfloat16 *)bias, (TOut *)phi, status, heads,
-                                                          (int)N);
+    npmap_tc_kernel<D, DF, TOut><<<grid, 192, kSmem, st>>>(tx, tw, (const __nv_bfloat16 *)bias, (TOut *)phi, csum, status, heads,
+                                                          (int)N, C);
     ++*launches;
     return cudaGetLastError() == cudaSuccess ? STILL_OK : STILL_ERR_CUDA;
 }
 
-template <typename TOut>
-int launch_npmap_any(const still_params_t *p, const void *X, const void *W, const void *bias, void *phi, int heads,
-                     long long N, int *status, cudaStream_t st, int *launches) {
-    if (p->d == 64 && p->d_f == 64) return launch_npmap<64, 64, TOut>(X, W, bias, phi, p->B, heads, N, status, st, launches);
-    if (p->d == 128 && p->d_f == 64) return launch_npmap<128, 64, TOut>(X, W, bias, phi, p->B, heads, N, status, st, launches);
-    if (p->d == 128 && p->d_f == 128) return launch_npmap<128, 128, TOut>(X, W, bias, phi, p->B, heads, N, status, st, launches);
-    return STILL_ERR_UNSUPPORTED;
-}
-
-template <int NF>
-int launch_scan(const still_params_t *p, long long N, const void *phiQ, const void *phiK, const void *V, const void *G,
-                const int32_t *sel_idx, float *nla, float *dla, float *S_out, float *z_out, int *status, cudaStream_t st,
-                int *launches) {
-    CUtensorMap tk, tv, tq;
+template <int D, int DF>
+int launch_fused(const still_params_t *p, long long N, const void *Q, const void *V, const void *G, const void *Wq,
+                 const void *bq, const int32_t *sel_idx, const void *phiK, const float *zpre, void *y_part, float *d_part,
+                 float *S_out, int *status, cudaStream_t st, int *launches) {
+    using bf = __nv_bfloat16;
+    CUtensorMap tq, tw, tk, tv;
     const unsigned long long BH = (unsigned long long)p->B * p->H, BHkv = (unsigned long long)p->B * p->Hkv;
-    if (!make_map_2d(&tk, phiK, BHkv * N, NF, 64, false) || !make_map_2d(&tv, V, BHkv * N, p->d, 64, false) ||
-        !make_map_2d(&tq, phiQ, BH * N, NF, 64, true))
+    if (!make_map_2d(&tq, Q, BH * N, D, 128, false) || !make_map_2d(&tw, Wq, (unsigned long long)p->H * D, DF, D, false) ||
+        !make_map_2d(&tk, phiK, BHkv * N, 2 * DF, 64, false) || !make_map_2d(&tv, V, BHkv * N, D, 64, false))
         return STILL_ERR_CUDA;
-    if (ensure_dynamic_smem((const void *)la_scan_tc_kernel<NF>, ScanPlan<NF>::kTotal) !=
-        cudaSuccess)
-        return STILL_ERR_CUDA;
-    dim3 grid((unsigned)BH, (unsigned)(p->d / 64));
-    la_scan_tc_kernel<NF><<<grid, 192, ScanPlan<NF>::kTotal, st>>>(tk, tv, tq, (const __nv_bfloat16 *)G, sel_idx, nla, dla,
-                                                                  S_out, z_out, status, p->H, p->Hkv, (int)N, p->d,
-                                                                  p->chunk, p->topk);
+    using Plan = FusedPlan<D, DF>;
+    if (ensure_dynamic_smem((const void *)la_fused_kernel<D, DF>, Plan::kTotal) != cudaSuccess) return STILL_ERR_CUDA;
+    dim3 grid((unsigned)BH, 2);   // the two feature halves of a head
+    la_fused_kernel<D, DF><<<grid, 384, Plan::kTotal, st>>>(tq, tw, tk, tv, (const bf *)bq, (const bf *)G, sel_idx, zpre, (bf *)y_part,
+                                                           d_part, S_out, status, p->H, p->Hkv, (int)N, p->chunk, p->topk,
+                                                           (long long)BH * N * D, (long long)BH * N);
     ++*launches;
     return cudaGetLastError() == cudaSuccess ? STILL_OK : STILL_ERR_CUDA;
 }
@@ -605,17 +848,40 @@ bool tc_la_supported(const still_params_t *p) {
 }
 
 int tc_la_branch(const still_params_t *p, long long N, const void *Q, const void *K, const void *V, const void *G,
-                 const void *Wq, const void *bq, const void *Wk, const void *bk, const int32_t *sel_idx, void *phiQ,
-                 void *phiK, float *nla, float *dla, float *S_out, float *z_out, int *status_words, cudaStream_t st,
-                 int *launches) {
+                 const void *Wq, const void *bq, const void *Wk, const void *bk, const int32_t *sel_idx, void *phiK,
+                 float *csum, float *zpre, void *y_part, float *d_part, float *S_out, float *z_out, int *status_words,
+                 cudaStream_t st, int *launches) {
+    using bf = __nv_bfloat16;
     if ((long long)p->B * p->H * N >= (1ll << 31)) return STILL_ERR_UNSUPPORTED;  // TMA row coordinate
-    int rc = launch_npmap_any<float>(p, Q, Wq, bq, phiQ, p->H, N, status_words, st, launches);
+    const int NF = 2 * p->d_f, C = p->chunk;
+    const long long Tn = (N + C - 1) / C, BH = (long long)p->B * p->H;
+    const int n_routed = Tn >= 3 ? (int)(Tn - 2) : 0;
+    // phi(K) once per KV head (bf16; the B operand of the state update), with the column sums of every chunk
+    int rc;
+    if (p->d == 64 && p->d_f == 64)
+        rc = launch_npmap<64, 64, bf>(K, Wk, bk, phiK, csum, p->B, p->Hkv, N, C, status_words, st, launches);
+    else if (p->d == 128 && p->d_f == 64)
+        rc = launch_npmap<128, 64, bf>(K, Wk, bk, phiK, csum, p->B, p->Hkv, N, C, status_words, st, launches);
+    else
+        rc = launch_npmap<128, 128, bf>(K, Wk, bk, phiK, csum, p->B, p->Hkv, N, C, status_words, st, launches);
     if (rc != STILL_OK) return rc;
-    rc = launch_npmap_any<__nv_bfloat16>(p, K, Wk, bk, phiK, p->Hkv, N, status_words, st, launches);
-    if (rc != STILL_OK) return rc;
-    if (p->d_f == 64)
-        return launch_scan<128>(p, N, phiQ, phiK, V, G, sel_idx, nla, dla, S_out, z_out, status_words, st, launches);
-    return launch_scan<256>(p, N, phiQ, phiK, V, G, sel_idx, nla, dla, S_out, z_out, status_words, st, launches);
+    // z after every routed chunk (per query head: the selection is per query head)
+    if (n_routed > 0) {
+        z_delta_kernel<<<dim3((unsigned)n_routed, (unsigned)BH), NF, 0, st>>>(csum, (const bf *)phiK, sel_idx, zpre, p->H, p->Hkv,
+                                                                                N, (int)Tn, n_routed, p->topk, NF);
+        ++*launches;
+        if (cudaGetLastError() != cudaSuccess) return STILL_ERR_CUDA;
+    }
+    if (n_routed > 0 || z_out != nullptr) {
+        z_scan_kernel<<<(unsigned)BH, NF, 0, st>>>(zpre, z_out, n_routed, NF);
+        ++*launches;
+        if (cudaGetLastError() != cudaSuccess) return STILL_ERR_CUDA;
+    }
+    if (p->d == 64 && p->d_f == 64)
+        return launch_fused<64, 64>(p, N, Q, V, G, Wq, bq, sel_idx, phiK, zpre, y_part, d_part, S_out, status_words, st, launches);
+    if (p->d == 128 && p->d_f == 64)
+        return launch_fused<128, 64>(p, N, Q, V, G, Wq, bq, sel_idx, phiK, zpre, y_part, d_part, S_out, status_words, st, launches);
+    return launch_fused<128, 128>(p, N, Q, V, G, Wq, bq, sel_idx, phiK, zpre, y_part, d_part, S_out, status_words, st, launches);
 }
 
 }  // namespace still

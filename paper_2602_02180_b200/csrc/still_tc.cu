@@ -109,8 +109,9 @@ template <int D, int kKStages, int kVStages, bool kPair, class StreamT>
 __device__ __forceinline__ void softmax_role(const StreamT &st, const int x, const int tile_row0, const uint32_t tmem_base,
                                              uint64_t *s_full, uint64_t *k_empty, uint64_t *v_empty, uint64_t *p_half,
                                              const uint32_t p_half_cluster, uint64_t *o_final, volatile int *abort_flag,
-                                             int *status, uint8_t *stage_tile, const float *__restrict__ N_LA,
-                                             const float *__restrict__ D_LA, __nv_bfloat16 *__restrict__ Y, const int bh,
+                                             int *status, uint8_t *stage_tile, const __nv_bfloat16 *__restrict__ y_part,
+                                             const float *__restrict__ d_part, const int n_parts, const long long part_stride_y,
+                                             const long long part_stride_d, __nv_bfloat16 *__restrict__ Y, const int bh,
                                              const int N, const int C, const int lam, const float scale_log2) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     auto col_s = [](int xx) -> uint32_t { return (uint32_t)xx * 128u; };
@@ -234,41 +235,50 @@ __device__ __forceinline__ void softmax_role(const StreamT &st, const int x, con
             ++n_seen;
         }
         // ---- epilogue: y = (O e^{m-ms} + e^{-ms} N_LA) / (l e^{m-ms} + e^{-ms} D_LA), ms = max(m, 0)
-        // A thread owns a row, but loads / stores in which every lane touches a different row cost a
-        // memory instruction per 16 bytes and row; so N_LA comes in and Y goes out through shared memory
-        // with 16 consecutive lanes per row.  The staging space is this warp's 32 rows of the tile's Q
-        // region (one row = D bf16 = 2 D bytes), free once the tile's last Q K^T has completed; 16-byte
-        // pieces are swizzled by the row so that row-wise and piece-wise accesses avoid bank conflicts.
+        // The linear branch arrives as up to two partial results (one per feature half): y_p = N_p / D_p as bf16
+        // and D_p, so N_LA = sum y_p D_p and D_LA = sum D_p.  A thread owns a row, but loads / stores in which
+        // every lane touches a different row cost a memory instruction per 16 bytes and row; so the y_p come in
+        // and Y goes out through shared memory with 16 consecutive lanes per row.  The staging space is this
+        // warp's 32 rows of the tile's Q region (one row = D bf16 = 2 D bytes: D / 2 columns of both parts), free
+        // once the tile's last Q K^T has completed; 16-byte pieces are swizzled by the row so that row-wise and
+        // piece-wise accesses avoid bank conflicts.
         if (ok) ok = mbar_wait(o_final + x, 0, abort_flag, status, 9);
         ok = __all_sync(0xffffffffu, ok);
         if (ok) {
             tc_fence_after();
             constexpr int kRowBytes = D * 2, kPieces = kRowBytes / 16;   // pieces of 16 bytes per staged row
+            constexpr int kPartPieces = kPieces / 2;                     // pieces of one part (D / 2 columns)
             uint8_t *stg = stage_tile + (warp & 3) * 32 * kRowBytes;
             const int t0 = tile_row0 + (warp & 3) * 32;                    // first row of this warp
-            float fs = 1.f, fl = 0.f, dla = 0.f;
-            if (D_LA != nullptr && t < N) {
-                dla = D_LA[(long long)bh * N + t];
+            float fs = 1.f, fa = 0.f, fb = 0.f, dla = 0.f;
+            if (n_parts > 0 && t < N) {
+                const float da = d_part[(long long)bh * N + t];
+                const float db = n_parts > 1 ? d_part[part_stride_d + (long long)bh * N + t] : 0.f;
+                dla = da + db;
                 if (dla > 0.f) {
                     const float m_nat = m_used * 0.6931471805599453f;
                     const float ms = fmaxf(m_nat, 0.f);
                     fs = __expf(m_nat - ms);
-                    fl = __expf(-ms);
+                    const float fl = __expf(-ms);
+                    fa = fl * da;
+                    fb = fl * db;
                 }
             }
-            const float inv = 1.f / (l_sum * fs + fl * dla);
-            const bool with_la = (D_LA != nullptr) && __any_sync(0xffffffffu, dla > 0.f);
+            const float inv = 1.f / (l_sum * fs + fa + fb);
+            const bool with_la = (n_parts > 0) && __any_sync(0xffffffffu, dla > 0.f);
             uint32_t out[D / 2];   // the row as packed bf16
 #pragma unroll
-            for (int hh = 0; hh < 2; ++hh) {   // halves of D / 2 columns: as fp32 they fill one staged row
+            for (int hh = 0; hh < 2; ++hh) {   // halves of D / 2 columns
                 if (with_la) {
                     __syncwarp();
 #pragma unroll
                     for (int it = 0; it < kPieces; ++it) {
                         const int id = it * 32 + lane, row = id / kPieces, c = id % kPieces;
+                        const int part = c / kPartPieces, cc = c % kPartPieces;
                         uint4 v = make_uint4(0, 0, 0, 0);
-                        if (t0 + row < N)
-                            v = *reinterpret_cast<const uint4 *>(N_LA + ((long long)bh * N + t0 + row) * D + hh * (D / 2) + c * 4);
+                        if (t0 + row < N && part < n_parts)
+                            v = *reinterpret_cast<const uint4 *>(y_part + part * part_stride_y + ((long long)bh * N + t0 + row) * D +
+                                                                 hh * (D / 2) + cc * 8);
                         *reinterpret_cast<uint4 *>(stg + row * kRowBytes + ((c ^ (row & (kPieces - 1))) << 4)) = v;
                     }
                     __syncwarp();
@@ -279,16 +289,22 @@ __device__ __forceinline__ void softmax_role(const StreamT &st, const int x, con
                     tmem_ld32(lane_addr + col_o(x) + hh * (D / 2) + q * 32, orow);
                     tmem_wait_ld();
 #pragma unroll
-                    for (int j4 = 0; j4 < 8; ++j4) {
-                        float4 nl = make_float4(0.f, 0.f, 0.f, 0.f);
-                        if (with_la)
-                            nl = *reinterpret_cast<const float4 *>(stg + lane * kRowBytes + (((q * 8 + j4) ^ (lane & (kPieces - 1))) << 4));
-                        const float a0 = fmaf(fl, nl.x, __uint_as_float(orow[4 * j4]) * fs);
-                        const float a1 = fmaf(fl, nl.y, __uint_as_float(orow[4 * j4 + 1]) * fs);
-                        const float a2 = fmaf(fl, nl.z, __uint_as_float(orow[4 * j4 + 2]) * fs);
-                        const float a3 = fmaf(fl, nl.w, __uint_as_float(orow[4 * j4 + 3]) * fs);
-                        out[hh * (D / 4) + q * 16 + 2 * j4] = pack_bf16(a0 * inv, a1 * inv);
-                        out[hh * (D / 4) + q * 16 + 2 * j4 + 1] = pack_bf16(a2 * inv, a3 * inv);
+                    for (int j8 = 0; j8 < 4; ++j8) {
+                        uint4 pa = make_uint4(0, 0, 0, 0), pb = pa;
+                        if (with_la) {
+                            const int ca = q * 4 + j8, cb = kPartPieces + ca;
+                            pa = *reinterpret_cast<const uint4 *>(stg + lane * kRowBytes + ((ca ^ (lane & (kPieces - 1))) << 4));
+                            pb = *reinterpret_cast<const uint4 *>(stg + lane * kRowBytes + ((cb ^ (lane & (kPieces - 1))) << 4));
+                        }
+                        const uint32_t wa[4] = {pa.x, pa.y, pa.z, pa.w}, wb[4] = {pb.x, pb.y, pb.z, pb.w};
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {   // two columns per 32-bit word
+                            const float la0 = fmaf(fa, __uint_as_float(wa[e] << 16), fb * __uint_as_float(wb[e] << 16));
+                            const float la1 = fmaf(fa, __uint_as_float(wa[e] & 0xffff0000u), fb * __uint_as_float(wb[e] & 0xffff0000u));
+                            const float a0 = fmaf(__uint_as_float(orow[8 * j8 + 2 * e]), fs, la0);
+                            const float a1 = fmaf(__uint_as_float(orow[8 * j8 + 2 * e + 1]), fs, la1);
+                            out[hh * (D / 4) + q * 16 + 4 * j8 + e] = pack_bf16(a0 * inv, a1 * inv);
+                        }
                     }
                 }
             }
@@ -314,8 +330,8 @@ template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                    const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_ksel,
-                   const __grid_constant__ CUtensorMap tm_vsel, const float *__restrict__ N_LA,
-                   const float *__restrict__ D_LA, __nv_bfloat16 *__restrict__ Y, int *status, int H, int Hkv,
+                   const __grid_constant__ CUtensorMap tm_vsel, const __nv_bfloat16 *__restrict__ y_part,
+                   const float *__restrict__ d_part, int n_parts, __nv_bfloat16 *__restrict__ Y, int *status, int H, int Hkv,
                    int N, int C, int lam, int sel_rows, int sel_identity, float scale_log2, int n_qblocks) {
     using P = SmemPlan<D>;
     extern __shared__ uint8_t smem_raw[];
@@ -529,8 +545,9 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         // ------------------------------------------------------------ softmax + epilogue
         const int x = (warp - 4) >> 2;                 // 0: tile A, 1: tile B
         softmax_role<D, P::kKStages, P::kVStages, false>(st, x, R0 + x * kBlockM, tmem_base, s_full, k_empty, v_empty, p_half, 0u,
-                                                         o_final, abort_flag, status, smem + P::kQ + x * P::kTileBytes, N_LA,
-                                                         D_LA, Y, bh, N, C, lam, scale_log2);
+                                                         o_final, abort_flag, status, smem + P::kQ + x * P::kTileBytes, y_part,
+                                                         d_part, n_parts, (long long)gridDim.y * N * D, (long long)gridDim.y * N,
+                                                         Y, bh, N, C, lam, scale_log2);
     }
     tc_fence_before();
     __syncthreads();
@@ -590,8 +607,8 @@ template <int D>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 sa_merge_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                      const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_ksel,
-                     const __grid_constant__ CUtensorMap tm_vsel, const float *__restrict__ N_LA,
-                     const float *__restrict__ D_LA, __nv_bfloat16 *__restrict__ Y, int *status, int H, int Hkv, int N,
+                     const __grid_constant__ CUtensorMap tm_vsel, const __nv_bfloat16 *__restrict__ y_part,
+                     const float *__restrict__ d_part, int n_parts, __nv_bfloat16 *__restrict__ Y, int *status, int H, int Hkv, int N,
                      int C, int lam, int sel_rows, int sel_identity, float scale_log2, int n_pairs) {
     using P = PairPlan<D>;
     extern __shared__ uint8_t smem_raw[];
@@ -823,8 +840,9 @@ sa_merge_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         const int x = (warp - 4) >> 2;                 // 0: tile A, 1: tile B
         softmax_role<D, P::kKStages, P::kVStages, true>(st, x, R0 + x * 2 * kBlockM + (int)rank * kBlockM, tmem_base, s_full,
                                                         k_empty, v_empty, p_half, mapa(smem_u32(p_half), 0), o_final,
-                                                        abort_flag, status, smem + P::kQ + x * P::kQTile, N_LA, D_LA, Y, bh, N,
-                                                        C, lam, scale_log2);
+                                                        abort_flag, status, smem + P::kQ + x * P::kQTile, y_part, d_part, n_parts,
+                                                        (long long)gridDim.y * N * D, (long long)gridDim.y * N, Y, bh, N, C, lam,
+                                                        scale_log2);
         if (*abort_flag) tell_peer();
     }
     // Nobody touches the peer's shared memory or tensor memory after this point.
@@ -1178,7 +1196,7 @@ bool make_map(CUtensorMap *m, const void *base, unsigned long long rows, int d) 
 
 template <int D>
 int launch_tc(const still_params_t *p, long long N, const void *Q, const void *K, const void *V,
-              const int32_t *sel_idx, const float *N_LA, const float *D_LA, void *Y, void *k_sel, void *v_sel,
+              const int32_t *sel_idx, const void *y_part, const float *d_part, int n_parts, void *Y, void *k_sel, void *v_sel,
               long long sel_rows, int *status, cudaStream_t st, int *launches) {
     using bf = __nv_bfloat16;
     const long long T = (N + p->chunk - 1) / p->chunk, BH = (long long)p->B * p->H;
@@ -1207,7 +1225,7 @@ int launch_tc(const still_params_t *p, long long N, const void *Q, const void *K
         dim3 grid((unsigned)(2 * n_pairs), (unsigned)BH);   // clusters of two along x
         profile_mark_begin(st);
         sa_merge_pair_kernel<D><<<grid, kThreads, PairPlan<D>::kAlloc, st>>>(
-            tq, tk, tv, tks, tvs, N_LA, D_LA, (bf *)Y, status, p->H, p->Hkv, (int)N, p->chunk, p->topk, (int)sel_rows,
+            tq, tk, tv, tks, tvs, (const bf *)y_part, d_part, n_parts, (bf *)Y, status, p->H, p->Hkv, (int)N, p->chunk, p->topk, (int)sel_rows,
             identity ? 1 : 0, scale_log2, n_pairs);
         profile_mark_end(st);
     } else {
@@ -1216,7 +1234,7 @@ int launch_tc(const still_params_t *p, long long N, const void *Q, const void *K
         dim3 grid((unsigned)n_qblocks, (unsigned)BH);
         profile_mark_begin(st);
         sa_merge_tc_kernel<D><<<grid, kThreads, SmemPlan<D>::kAlloc, st>>>(
-            tq, tk, tv, tks, tvs, N_LA, D_LA, (bf *)Y, status, p->H, p->Hkv, (int)N, p->chunk, p->topk, (int)sel_rows,
+            tq, tk, tv, tks, tvs, (const bf *)y_part, d_part, n_parts, (bf *)Y, status, p->H, p->Hkv, (int)N, p->chunk, p->topk, (int)sel_rows,
             identity ? 1 : 0, scale_log2, n_qblocks);
         profile_mark_end(st);
     }
@@ -1262,6 +1280,25 @@ int tc_score_select(const still_params_t *p, long long N, const void *Q, const v
     return launch_score_tc<128, 128>(p, N, Q, K, scores, sel_idx, status_words, st, launches);
 }
 
+// N_LA / D_LA of the fp32-accumulating FMA kernels as one bf16 part: y = N_LA / D_LA, d = D_LA.
+__global__ void la_to_part_kernel(const float *__restrict__ N_LA, const float *__restrict__ D_LA, __nv_bfloat16 *__restrict__ y,
+                                  float *__restrict__ dp, long long rows, int d) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= rows * d) return;
+    const long long r = i / d;
+    const float dd = D_LA[r];
+    y[i] = __float2bfloat16_rn(dd > 0.f ? N_LA[i] / dd : 0.f);
+    if (i == r * d) dp[r] = dd;
+}
+
+int tc_la_to_part(const float *N_LA, const float *D_LA, void *y_part, float *d_part, long long rows, int d, cudaStream_t st,
+                  int *launches) {
+    const long long n = rows * d;
+    la_to_part_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(N_LA, D_LA, (__nv_bfloat16 *)y_part, d_part, rows, d);
+    ++*launches;
+    return cudaGetLastError() == cudaSuccess ? STILL_OK : STILL_ERR_CUDA;
+}
+
 int tc_selftest_wait_timeout(int *status_words, long long limit_cycles, cudaStream_t st) {
     wait_timeout_selftest_kernel<<<1, 32, 0, st>>>(status_words, limit_cycles);
     return cudaGetLastError() == cudaSuccess ? STILL_OK : STILL_ERR_CUDA;
@@ -1277,12 +1314,12 @@ long long tc_sel_rows(const still_params_t *p, long long N) {
 }
 
 int tc_sa_merge(const still_params_t *p, long long N, const void *Q, const void *K, const void *V,
-                const int32_t *sel_idx, const float *N_LA, const float *D_LA, void *Y, void *k_sel, void *v_sel,
+                const int32_t *sel_idx, const void *y_part, const float *d_part, int n_parts, void *Y, void *k_sel, void *v_sel,
                 long long sel_rows, int *status_words, cudaStream_t st, int *launches) {
     if ((long long)p->B * p->H * std::max(N, sel_rows) >= (1ll << 31)) return STILL_ERR_UNSUPPORTED;  // TMA row coordinate
     if (p->d == 64)
-        return launch_tc<64>(p, N, Q, K, V, sel_idx, N_LA, D_LA, Y, k_sel, v_sel, sel_rows, status_words, st, launches);
-    return launch_tc<128>(p, N, Q, K, V, sel_idx, N_LA, D_LA, Y, k_sel, v_sel, sel_rows, status_words, st, launches);
+        return launch_tc<64>(p, N, Q, K, V, sel_idx, y_part, d_part, n_parts, Y, k_sel, v_sel, sel_rows, status_words, st, launches);
+    return launch_tc<128>(p, N, Q, K, V, sel_idx, y_part, d_part, n_parts, Y, k_sel, v_sel, sel_rows, status_words, st, launches);
 }
 
 }  // namespace still

@@ -41,9 +41,14 @@ long long tc_sel_rows(const still_params_t *p, long long N);
 int tc_score_select(const still_params_t *p, long long N, const void *Q, const void *K, float *scores,
                     int32_t *sel_idx, int *status_words, cudaStream_t st, int *launches);
 // Compacts the selected K/V rows and runs the softmax-attention + merge kernel.
+// The linear branch arrives as n_parts (0, 1 or 2) partial results: y_part [n_parts][B,H,N,d] bf16 = N_part /
+// D_part and d_part [n_parts][B,H,N] fp32; N_LA = sum y_part d_part, D_LA = sum d_part.
 int tc_sa_merge(const still_params_t *p, long long N, const void *Q, const void *K, const void *V,
-                const int32_t *sel_idx, const float *N_LA, const float *D_LA, void *Y, void *k_sel,
+                const int32_t *sel_idx, const void *y_part, const float *d_part, int n_parts, void *Y, void *k_sel,
                 void *v_sel, long long sel_rows, int *status_words, cudaStream_t st, int *launches);
+// fp32 N_LA / D_LA of the FMA kernels as one such part (y = N_LA / D_LA, d = D_LA).
+int tc_la_to_part(const float *N_LA, const float *D_LA, void *y_part, float *d_part, long long rows, int d,
+                  cudaStream_t st, int *launches);
 
 // One CTA whose only act is a bounded mbarrier wait on a barrier that nothing arrives on: the wait runs
 // out after limit_cycles, the kernel records STILL_ERR_DEVICE_TIMEOUT (detail 99) in status_words and
@@ -53,13 +58,14 @@ int tc_selftest_wait_timeout(int *status_words, long long limit_cycles, cudaStre
 // ---- tensor-core linear-attention branch of the prefill, bf16 only --------------------
 // True when NP-Map and the chunk-wise state scan of these parameters run on the tcgen05 kernels.
 bool tc_la_supported(const still_params_t *p);
-// NP-Map of Q (fp32 features into phiQ [B,H,N,2 d_f]) and of K (bf16 features into phiK
-// [B,Hkv,N,2 d_f]), then the state scan: N_LA [B,H,N,d] (gated), D_LA [B,H,N]; S_out / z_out
-// (optional) receive the state after the chunks that have left the local region.
+// NP-Map of K (bf16 features into phiK [B,Hkv,N,2 d_f], chunk column sums into csum [B,Hkv,T,2 d_f]), the
+// normaliser z after every routed chunk (zpre [B,H,T-2,2 d_f]), then the state scan with the query-side NP-Map
+// fused in: y_part [2][B,H,N,d] bf16 = N_part / D_part (gated), d_part [2][B,H,N] fp32, one part per feature
+// half; S_out / z_out (optional) receive the state after the chunks that have left the local region.
 int tc_la_branch(const still_params_t *p, long long N, const void *Q, const void *K, const void *V, const void *G,
-                 const void *Wq, const void *bq, const void *Wk, const void *bk, const int32_t *sel_idx, void *phiQ,
-                 void *phiK, float *nla, float *dla, float *S_out, float *z_out, int *status_words, cudaStream_t st,
-                 int *launches);
+                 const void *Wq, const void *bq, const void *Wk, const void *bk, const int32_t *sel_idx, void *phiK,
+                 float *csum, float *zpre, void *y_part, float *d_part, float *S_out, float *z_out, int *status_words,
+                 cudaStream_t st, int *launches);
 
 // ---- decode step ----------------------------------------------------------------------
 size_t step_scratch_bytes(const still_params_t *p, long long capacity);

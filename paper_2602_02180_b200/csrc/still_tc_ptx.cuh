@@ -140,6 +140,28 @@ __device__ __forceinline__ void mma_ss_lo(uint32_t d_tmem, uint32_t a_lo, uint32
         ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(kDescHi), "r"(kIdesc), "n"(kAcc)
         : "memory");
 }
+// D[tmem] (+)= A[smem] * B[smem] with a run-time accumulate flag.
+template <uint32_t kIdesc>
+__device__ __forceinline__ void mma_ss_lo_acc(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(kDescHi), "r"(kIdesc), "r"(acc)
+        : "memory");
+}
+// D[tmem] (+)= A[tmem, fp32 read as TF32] * B[smem]; kAcc = 0 overwrites D.
+template <uint32_t kIdesc, uint32_t kAcc>
+__device__ __forceinline__ void mma_ts_tf32_lo(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], db, %4, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(kDescHi), "r"(kIdesc), "n"(kAcc)
+        : "memory");
+}
 // D[tmem] (+)= A[tmem] * B[smem]; acc = 0 overwrites D.
 template <uint32_t kIdesc>
 __device__ __forceinline__ void mma_ts_lo(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t acc) {
