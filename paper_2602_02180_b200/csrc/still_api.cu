@@ -52,7 +52,7 @@ static inline bool la_active(const still_params_t *p) { return p->topk < p->chun
 
 // Workspace plan of the prefill.
 struct FwdPlan {
-    size_t status, scores, sel_idx, phiQ, phiK, csum, zpre, nla, dla, ypart, dpart, ksel, vsel, total;
+    size_t status, scores, sel_idx, phiQ, phiK, csum, zpre, segs, nla, dla, ypart, dpart, ksel, vsel, total;
     long long T, sel_rows;  // chunks; rows of the compacted salient K/V per head
     bool la, tc, tc_la;
 };
@@ -81,6 +81,7 @@ static FwdPlan plan_fwd(const still_params_t *p, long long N) {
             // tensor-core branch: phi(Q) is never stored; the branch leaves two bf16 partial results
             w.csum = take(BHkv * (size_t)T * dp * 4);
             w.zpre = take(BH * (size_t)std::max<long long>(T - 2, 1) * dp * 4);
+            w.segs = take(BH * (size_t)std::max(tc_la_segments(p, N, nullptr) - 1, 1) * dp * p->d * 4);
         } else {
             w.phiQ = take(BH * (size_t)N * dp * es);
             w.nla = take(BH * (size_t)N * p->d * 4);
@@ -295,7 +296,8 @@ static int fwd_typed(const still_params_t *p, long long N, const T *Q, const T *
             dpart = reinterpret_cast<float *>(ws + w.dpart);
             n_parts = 2;
             rc = tc_la_branch(p, N, Q, K, V, G, Wq, bq, Wk, bk, sel, phiK, reinterpret_cast<float *>(ws + w.csum),
-                              reinterpret_cast<float *>(ws + w.zpre), ypart, dpart, S_out, z_out,
+                              reinterpret_cast<float *>(ws + w.zpre), ypart, dpart, reinterpret_cast<float *>(ws + w.segs), S_out,
+                              z_out,
                               reinterpret_cast<int *>(ws + w.status), st, &g_launches);
             if (rc != STILL_OK) return rc;
         } else {

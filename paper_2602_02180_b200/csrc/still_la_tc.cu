@@ -351,15 +351,15 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 const __grid_constant__ CUtensorMap tm_phik, const __grid_constant__ CUtensorMap tm_v,
                 const __nv_bfloat16 *__restrict__ bq, const __nv_bfloat16 *__restrict__ G,
                 const int32_t *__restrict__ sel_idx, const float *__restrict__ zpre, __nv_bfloat16 *__restrict__ y_part,
-                float *__restrict__ d_part, float *__restrict__ S_out, int *status, int H, int Hkv, int N, int C, int lam,
-                long long part_stride_y, long long part_stride_d) {
+                float *__restrict__ d_part, float *__restrict__ S_out, float *__restrict__ seg_sums, int *status, int H, int Hkv,
+                int N, int C, int lam, long long part_stride_y, long long part_stride_d, int seg_chunks, int n_seg, int sums_only) {
     using P = FusedPlan<D, DF>;
     constexpr int NF = 2 * DF;
     extern __shared__ __align__(1024) uint8_t smem[];
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + P::oBar);
     uint64_t *w_full = bars, *x_full = bars + 1, *x_empty = bars + 2, *f_done = bars + 3, *f_free = bars + 4;
     uint64_t *pq_full = bars + 5, *pq_empty = bars + 7, *u_full = bars + 9, *u_empty = bars + 11, *u_masked = bars + 13;
-    uint64_t *r_done = bars + 15, *out_free = bars + 17, *fin = bars + 19;
+    uint64_t *r_done = bars + 15, *out_free = bars + 17, *fin = bars + 19, *init_done = bars + 20;
     uint32_t *tmem_base_slot = reinterpret_cast<uint32_t *>(smem + P::oMisc);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + P::oMisc + 8);
     float *dinv_ring = reinterpret_cast<float *>(smem + P::oDinv);
@@ -369,12 +369,19 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const int half = blockIdx.y;                // 0: features softmax(u), 1: features softmax(-u)
     const int sc = C / 64;                      // 64-token sub-chunks per chunk
     const int Tn = (N + C - 1) / C;
-    const int NU = (N + 63) / 64;               // sub-chunks with query rows
-    const int NB = (N + 127) / 128;             // blocks of 128 query rows
     const int n_routed = Tn >= 3 ? Tn - 2 : 0;  // chunks whose tokens enter the state
-    const int n_upd = n_routed * sc;            // update tiles (sub-chunks of the routed chunks)
-    const int u_first = 2 * sc;                 // first sub-chunk whose read-out sees a non-empty state
-    const int b_first = u_first / 2;            // its block
+    // The sequence is cut into n_seg segments of seg_chunks chunks (two-level scan): segment g answers the
+    // sub-chunks [u_first, NU) and performs the updates that fall between them, starting from the sum of the
+    // earlier segments' updates (seg_sums, produced by a first pass of this kernel with sums_only set).
+    const int seg = blockIdx.z;
+    const int NU_all = (N + 63) / 64;           // sub-chunks with query rows
+    const int u_first = seg == 0 ? 2 * sc : seg * seg_chunks * sc;   // the first two chunks see an empty state
+    const int NU = (!sums_only && seg == n_seg - 1) ? NU_all : min(NU_all, (seg + 1) * seg_chunks * sc);
+    const int b_first = u_first / 2;            // blocks of 128 query rows: [b_first, NB)
+    const int NB = sums_only ? b_first : (NU + 1) / 2;
+    const int nu0 = (u_first / sc - 2) * sc;    // first update tile of the segment (64-token sub-chunks of routed chunks)
+    const int n_upd = NU > u_first ? ((NU - 1) / sc - 1) * sc - nu0 : 0;
+    const bool has_init = !sums_only && seg > 0;
     __nv_bfloat16 *y_out = y_part + (long long)half * part_stride_y;
     float *d_out = d_part + (long long)half * part_stride_d;
 
@@ -402,6 +409,7 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             mbar_init(out_free + i, 4);
         }
         mbar_init(fin, 1);
+        mbar_init(init_done, 4);
         *abort_flag = 0;
         fence_barrier_init();
     }
@@ -445,9 +453,9 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     uint8_t *stg = smem + P::oU + (nu & 1) * P::kUStage;
                     mbar_expect_tx(u_full + (nu & 1), P::kUStage);
                     for (int a = 0; a < DF / 64; ++a)  // phi(K) half: MN-major, 64-feature atoms 64 rows apart
-                        tma_load_2d(stg + a * (64 * 128), &tm_phik, u_full + (nu & 1), half * DF + a * 64, kv_row0 + nu * 64);
+                        tma_load_2d(stg + a * (64 * 128), &tm_phik, u_full + (nu & 1), half * DF + a * 64, kv_row0 + (nu0 + nu) * 64);
                     for (int a = 0; a < D / 64; ++a)   // V: M-major A operand, 64-column atoms 64 rows apart
-                        tma_load_2d(stg + P::kPhiK + a * (64 * 128), &tm_v, u_full + (nu & 1), a * 64, kv_row0 + nu * 64);
+                        tma_load_2d(stg + P::kPhiK + a * (64 * 128), &tm_v, u_full + (nu & 1), a * 64, kv_row0 + (nu0 + nu) * 64);
                     ++nu;
                     progressed = true;
                 }
@@ -499,21 +507,29 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 ++nx;
                 return true;
             };
-            if (NB > b_first) ok = issue_f();
-            for (int u = u_first; u < NU && ok; ++u) {
+            if (has_init) {   // the workers have put the sum of the earlier segments into tensor memory
+                ok = mbar_wait(init_done, 0, abort_flag, status, 73);
+                tc_fence_after();
+            }
+            auto issue_update = [&]() -> bool {
+                if (!mbar_wait(u_masked + (nu & 1), (nu >> 1) & 1, abort_flag, status, 64)) return false;
+                tc_fence_after();
+                const uint32_t so = (uint32_t)(nu & 1) * (P::kUStage >> 4);
+#pragma unroll
+                for (int k = 0; k < 4; ++k)   // 16 tokens per step: 16 rows of 128 bytes in both operands
+                    mma_ss_lo_acc<idesc_upd>(tmem_base + col_state, v_lo0 + so + k * (2048 >> 4), pk_lo0 + so + k * (2048 >> 4),
+                                             (nu > 0 || k > 0 || has_init) ? 1u : 0u);
+                tc_commit(u_empty + (nu & 1));
+                ++nu;
+                return true;
+            };
+            if (sums_only)
+                while (ok && nu < n_upd) ok = issue_update();
+            if (ok && NB > b_first) ok = issue_f();
+            for (int u = u_first; u < NU && ok && !sums_only; ++u) {
                 if (u % sc == 0) {
                     // the chunk that has just left the local region: sub-chunks of chunk u / sc - 2
-                    for (int j = 0; j < sc && ok; ++j, ++nu) {
-                        ok = mbar_wait(u_masked + (nu & 1), (nu >> 1) & 1, abort_flag, status, 64);
-                        if (!ok) break;
-                        tc_fence_after();
-                        const uint32_t so = (uint32_t)(nu & 1) * (P::kUStage >> 4);
-#pragma unroll
-                        for (int k = 0; k < 4; ++k)   // 16 tokens per step: 16 rows of 128 bytes in both operands
-                            mma_ss_lo_acc<idesc_upd>(tmem_base + col_state, v_lo0 + so + k * (2048 >> 4), pk_lo0 + so + k * (2048 >> 4),
-                                                     (nu > 0 || k > 0) ? 1u : 0u);
-                        tc_commit(u_empty + (nu & 1));
-                    }
+                    for (int j = 0; j < sc && ok; ++j) ok = issue_update();
                     if (!ok) break;
                 }
                 ok = mbar_wait(pq_full + (u & 1), (nq >> 1) & 1, abort_flag, status, 65);
@@ -545,7 +561,7 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         // state.  The chunk's indices are fetched before the tile is waited for.
         bool ok = true;
         for (int nu = 0; nu < n_upd; ++nu) {
-            const int chunk = nu / sc, sub = nu % sc;
+            const int chunk = (nu0 + nu) / sc, sub = (nu0 + nu) % sc;
             const int32_t *si = sel_idx + ((long long)bh * Tn + chunk) * lam;
             int row[4];
 #pragma unroll
@@ -581,13 +597,33 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         bool ok = true;
         int nq = 0;
         // rows of the first two chunks see an empty state
-        {
-            const int n0 = min(N, u_first * 64);
+        if (seg == 0 && !sums_only) {
+            const int n0 = min(N, 2 * C);
             for (int i = tid; i < n0 * (D / 8); i += 128)
                 reinterpret_cast<uint4 *>(y_out + (long long)bh * N * D)[i] = make_uint4(0, 0, 0, 0);
             for (int t = tid; t < n0; t += 128) d_out[(long long)bh * N + t] = 0.f;
         }
-        for (int u = u_first; u < NU; ++u) {
+        if (has_init) {
+            // S^T of this segment starts as the sum of the earlier segments' updates: lane e, column f <- sum_g P_g[f][e]
+            const float *P0 = seg_sums + (((long long)bh * 2 + half) * (n_seg - 1)) * (DF * D);
+#pragma unroll 1
+            for (int q = 0; q < DF / 32; ++q) {
+                uint32_t sreg[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    float acc = 0.f;
+                    if (e < D)
+                        for (int g2 = 0; g2 < seg; ++g2) acc += P0[(long long)g2 * (DF * D) + (q * 32 + j) * D + e];
+                    sreg[j] = __float_as_uint(acc);
+                }
+                tmem_st32(taddr + col_state + q * 32, sreg);
+            }
+            tmem_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(init_done);
+        }
+        for (int u = u_first; u < NU && !sums_only; ++u) {
             if (ok) ok = mbar_wait(r_done + (nq & 1), (nq >> 1) & 1, abort_flag, status, 68);
             ok = __all_sync(0xffffffffu, ok);
             if (ok) {
@@ -646,9 +682,13 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             asm volatile("bar.sync 2, 128;" ::: "memory");   // the staging tile has been read before the next one is written
             ++nq;
         }
-        // final state for the decode state: S [2 d_f, d], this CTA's features
-        if (S_out != nullptr) {
-            if (n_upd > 0) {
+        // the state after the segment's last update: the segment's own sum for the second pass (sums_only), or,
+        // from the last segment, S [2 d_f, d] of the decode state (this CTA's features)
+        float *S_dst = nullptr;
+        if (sums_only) S_dst = seg_sums + (((long long)bh * 2 + half) * (n_seg - 1) + seg) * (DF * D);
+        else if (S_out != nullptr && seg == n_seg - 1) S_dst = S_out + ((long long)bh * NF + half * DF) * D;
+        if (S_dst != nullptr) {
+            if (n_upd > 0 || has_init) {
                 if (ok) ok = mbar_wait(fin, 0, abort_flag, status, 69);
                 ok = __all_sync(0xffffffffu, ok);
                 if (ok) {
@@ -660,13 +700,12 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         tmem_wait_ld();
                         if (e < D) {
 #pragma unroll
-                            for (int j = 0; j < 32; ++j)
-                                S_out[((long long)bh * NF + half * DF + q * 32 + j) * D + e] = __uint_as_float(sreg[j]);
+                            for (int j = 0; j < 32; ++j) S_dst[(q * 32 + j) * D + e] = __uint_as_float(sreg[j]);
                         }
                     }
                 }
             } else {
-                for (int i = tid; i < DF * D; i += 128) S_out[((long long)bh * NF + half * DF) * D + i] = 0.f;
+                for (int i = tid; i < DF * D; i += 128) S_dst[i] = 0.f;
             }
         }
     } else {
@@ -824,7 +863,7 @@ int launch_npmap(const void *X, const void *W, const void *bias, void *phi, floa
 template <int D, int DF>
 int launch_fused(const still_params_t *p, long long N, const void *Q, const void *V, const void *G, const void *Wq,
                  const void *bq, const int32_t *sel_idx, const void *phiK, const float *zpre, void *y_part, float *d_part,
-                 float *S_out, int *status, cudaStream_t st, int *launches) {
+                 float *S_out, float *seg_sums, int *status, cudaStream_t st, int *launches) {
     using bf = __nv_bfloat16;
     CUtensorMap tq, tw, tk, tv;
     const unsigned long long BH = (unsigned long long)p->B * p->H, BHkv = (unsigned long long)p->B * p->Hkv;
@@ -833,12 +872,19 @@ int launch_fused(const still_params_t *p, long long N, const void *Q, const void
         return STILL_ERR_CUDA;
     using Plan = FusedPlan<D, DF>;
     if (ensure_dynamic_smem((const void *)la_fused_kernel<D, DF>, Plan::kTotal) != cudaSuccess) return STILL_ERR_CUDA;
-    dim3 grid((unsigned)BH, 2);   // the two feature halves of a head
-    la_fused_kernel<D, DF><<<grid, 384, Plan::kTotal, st>>>(tq, tw, tk, tv, (const bf *)bq, (const bf *)G, sel_idx, zpre, (bf *)y_part,
-                                                           d_part, S_out, status, p->H, p->Hkv, (int)N, p->chunk, p->topk,
-                                                           (long long)BH * N * D, (long long)BH * N);
-    ++*launches;
-    return cudaGetLastError() == cudaSuccess ? STILL_OK : STILL_ERR_CUDA;
+    int seg_chunks = 0;
+    const int n_seg = tc_la_segments(p, N, &seg_chunks);
+    for (int pass = n_seg > 1 ? 0 : 1; pass < 2; ++pass) {
+        // pass 0 (only with several segments): the sum of every segment's own updates; pass 1: the scan proper
+        dim3 grid((unsigned)BH, 2, (unsigned)(pass == 0 ? n_seg - 1 : n_seg));   // head, feature half, segment
+        la_fused_kernel<D, DF><<<grid, 384, Plan::kTotal, st>>>(tq, tw, tk, tv, (const bf *)bq, (const bf *)G, sel_idx, zpre,
+                                                               (bf *)y_part, d_part, S_out, seg_sums, status, p->H, p->Hkv, (int)N,
+                                                               p->chunk, p->topk, (long long)BH * N * D, (long long)BH * N,
+                                                               seg_chunks, n_seg, pass == 0 ? 1 : 0);
+        ++*launches;
+        if (cudaGetLastError() != cudaSuccess) return STILL_ERR_CUDA;
+    }
+    return STILL_OK;
 }
 
 }  // namespace
@@ -847,10 +893,23 @@ bool tc_la_supported(const still_params_t *p) {
     return tc_supported(p) && (p->d_f == 64 || p->d_f == 128) && p->d_f <= p->d;
 }
 
+// Two-level scan: with few (batch, head) units the sequence is cut into segments that run side by side, each
+// starting from the sum of the earlier segments' state updates.  Segments are whole, even numbers of chunks, at
+// least eight of them, and as many as fill the SMs once (two CTAs per head and segment).
+int tc_la_segments(const still_params_t *p, long long N, int *seg_chunks) {
+    const long long Tn = (N + p->chunk - 1) / p->chunk, ctas = 2ll * p->B * p->H;
+    int n_seg = 1;
+    while (n_seg < 4 && ctas * (n_seg * 2) <= 148 && Tn / (n_seg * 2) >= 8) n_seg *= 2;
+    long long sc = (Tn + n_seg - 1) / n_seg;
+    sc += sc & 1;
+    if (seg_chunks) *seg_chunks = (int)sc;
+    return n_seg;
+}
+
 int tc_la_branch(const still_params_t *p, long long N, const void *Q, const void *K, const void *V, const void *G,
                  const void *Wq, const void *bq, const void *Wk, const void *bk, const int32_t *sel_idx, void *phiK,
-                 float *csum, float *zpre, void *y_part, float *d_part, float *S_out, float *z_out, int *status_words,
-                 cudaStream_t st, int *launches) {
+                 float *csum, float *zpre, void *y_part, float *d_part, float *seg_sums, float *S_out, float *z_out,
+                 int *status_words, cudaStream_t st, int *launches) {
     using bf = __nv_bfloat16;
     if ((long long)p->B * p->H * N >= (1ll << 31)) return STILL_ERR_UNSUPPORTED;  // TMA row coordinate
     const int NF = 2 * p->d_f, C = p->chunk;
@@ -878,10 +937,10 @@ int tc_la_branch(const still_params_t *p, long long N, const void *Q, const void
         if (cudaGetLastError() != cudaSuccess) return STILL_ERR_CUDA;
     }
     if (p->d == 64 && p->d_f == 64)
-        return launch_fused<64, 64>(p, N, Q, V, G, Wq, bq, sel_idx, phiK, zpre, y_part, d_part, S_out, status_words, st, launches);
+        return launch_fused<64, 64>(p, N, Q, V, G, Wq, bq, sel_idx, phiK, zpre, y_part, d_part, S_out, seg_sums, status_words, st, launches);
     if (p->d == 128 && p->d_f == 64)
-        return launch_fused<128, 64>(p, N, Q, V, G, Wq, bq, sel_idx, phiK, zpre, y_part, d_part, S_out, status_words, st, launches);
-    return launch_fused<128, 128>(p, N, Q, V, G, Wq, bq, sel_idx, phiK, zpre, y_part, d_part, S_out, status_words, st, launches);
+        return launch_fused<128, 64>(p, N, Q, V, G, Wq, bq, sel_idx, phiK, zpre, y_part, d_part, S_out, seg_sums, status_words, st, launches);
+    return launch_fused<128, 128>(p, N, Q, V, G, Wq, bq, sel_idx, phiK, zpre, y_part, d_part, S_out, seg_sums, status_words, st, launches);
 }
 
 }  // namespace still

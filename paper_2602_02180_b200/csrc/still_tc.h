@@ -64,8 +64,11 @@ bool tc_la_supported(const still_params_t *p);
 // half; S_out / z_out (optional) receive the state after the chunks that have left the local region.
 int tc_la_branch(const still_params_t *p, long long N, const void *Q, const void *K, const void *V, const void *G,
                  const void *Wq, const void *bq, const void *Wk, const void *bk, const int32_t *sel_idx, void *phiK,
-                 float *csum, float *zpre, void *y_part, float *d_part, float *S_out, float *z_out, int *status_words,
-                 cudaStream_t st, int *launches);
+                 float *csum, float *zpre, void *y_part, float *d_part, float *seg_sums, float *S_out, float *z_out,
+                 int *status_words, cudaStream_t st, int *launches);
+// Segments of the two-level state scan for these parameters (1 = plain scan); *seg_chunks = chunks per segment.
+// seg_sums holds (segments - 1) partial states [2 d_f, d] fp32 per (batch, head).
+int tc_la_segments(const still_params_t *p, long long N, int *seg_chunks);
 
 // ---- decode step ----------------------------------------------------------------------
 size_t step_scratch_bytes(const still_params_t *p, long long capacity);

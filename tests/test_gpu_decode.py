@@ -105,6 +105,7 @@ def _decode_case(w, n0, n_steps, gate=False, tweak=None, expect_ties=False, n_he
         (1, 2, 2, 128, 128, 32, 300, 90),
         (1, 16, 1, 64, 32, 8, 90, 50),     # sixteen query heads on one KV head
         (1, 12, 2, 128, 64, 16, 200, 70),  # six heads per group
+        (1, 2, 1, 128, 64, 16, 64 * 36 + 5, 70),   # long prefill on few heads: the state comes out of a segmented scan
     ],
 )
 def test_decode_matches_oracle(dtype, B, H, Hkv, d, C, k, n0, steps):

@@ -38,6 +38,8 @@ def test_c1_fp32_every_row():
         (1, 1, 1, 64, 1, 32, 4),        # a single token
         (1, 8, 2, 128, 128 * 4, 128, 128),
         (1, 4, 2, 64, 128 * 3 + 70, 128, 32),   # d = 64 with C = 128: two 64-token sub-chunks per chunk
+        (1, 2, 1, 128, 64 * 40 + 17, 64, 16),   # many chunks, few heads: the state scan runs as four segments
+        (1, 2, 2, 64, 128 * 33 + 5, 128, 32),   # the same with two sub-chunks per chunk (two segments)
     ],
 )
 def test_small_shapes(dtype, B, H, Hkv, d, N, C, k):
