@@ -183,6 +183,32 @@ def oracle_decode_sample(w, lam, n_rows=257):
                       f"the {w.N}-token prefix (prefix work excluded), scaled by head count"}
 
 
+def local_global_overlap(w, n_tokens=4096, n_heads=4):
+    """Sec. 3.1's local-global consistency on the synthetic inputs (CPU oracle): how much of each chunk's top-C/4 by
+    the windowed Self-Saliency Score is also in its top-C/4 by the full-context score.  Bounded: the first n_tokens
+    tokens of n_heads heads (the full-context score costs O(N^2 d) per head)."""
+    import numpy as np
+
+    from oracle import still_oracle as oracle
+    from paper_2602_02180_b200 import synth
+
+    n = min(n_tokens, w.N)
+    ws = w.with_(B=1, H=n_heads, Hkv=n_heads, N=n)
+    Q, K, _ = synth.make_qkv(ws, "cpu")
+    lam = max(w.C // 4, 1)
+    hits = []
+    for h in range(n_heads):
+        q, k = (t[0, h].float().numpy().astype(np.float64) for t in (Q, K))
+        loc = oracle.select(oracle.score_chunkwise(q, k, w.C, w.sm_scale), w.C, lam)
+        glo = oracle.select(oracle.score_global(q, k, w.sm_scale), w.C, lam)
+        for a, b in zip(loc, glo):
+            sa, sb = set(a[a >= 0].tolist()), set(b[b >= 0].tolist())
+            if sa:
+                hits.append(len(sa & sb) / len(sa))
+    return {"workload": w.name, "tokens": n, "heads": n_heads, "chunk": w.C, "topk": lam,
+            "mean_overlap": float(np.mean(hits)), "min_overlap": float(np.min(hits))}
+
+
 def run_reference(args, w, lam, rank, world):
     """--impl reference: the CPU oracle as it stands, on this machine's host cores."""
     if rank != 0:
@@ -435,6 +461,8 @@ def bench_prefill(args, w, lam, still, synth, torch, dist, dev, rank, world):
         n_heads = max(1, min(multiprocessing.cpu_count(), w.B * w.H))
         total, threads, sample, _ = oracle_sample(w, lam, n_heads, 160 if w.N > 8192 else 256)
         cpu = {"value": w.B * w.N / total, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample}
+        if companions is not None:
+            cpu["local_vs_global_selection"] = [local_global_overlap(synth.WORKLOADS[n]) for n in ("c2", "c3", "c4")]
 
     return {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,

@@ -95,6 +95,13 @@ def score_tokenwise(q, k, w, sm_scale, eps=1e-6):
     return out
 
 
+def score_global(q, k, sm_scale, eps=1e-6):
+    """Self-Saliency Score with the full causal context as the window, W_t = {1..t}: the global variant the
+    local score is compared with in Sec. 3.1 (local-global consistency).  It is the window-set definition with
+    a window that is never shorter than the prefix."""
+    return score_tokenwise(q, k, max(int(np.asarray(q).shape[0]), 1), sm_scale, eps)
+
+
 def score_chunkwise(q, k, C, sm_scale, eps=1e-6):
     """Self-Saliency Score from chunk tiles and masks (Algorithm 1)."""
     q, k = _f64(q), _f64(k)

@@ -95,6 +95,23 @@ def test_score_two_formulations_agree():
         )
 
 
+def test_global_score_is_the_window_score_with_an_unbounded_window():
+    # Sec. 3.1 compares the local score with its full-context variant, W_t = {1..t}.  While the sequence is no
+    # longer than the window the two coincide (token-wise and chunk-wise forms alike); beyond that they differ;
+    # with equal logits the global score of token t is the closed form for a window of t tokens.
+    N, d, C = 24, 6, 32
+    q, k, _, _, _ = _rand_head(N, d)
+    g = o.score_global(q, k, 0.4)
+    np.testing.assert_allclose(g, o.score_tokenwise(q, k, C, 0.4), rtol=1e-12)
+    np.testing.assert_allclose(g, o.score_chunkwise(q, k, C, 0.4), rtol=1e-10)
+    short = o.score_tokenwise(q, k, 8, 0.4)
+    np.testing.assert_allclose(g[:8], short[:8], rtol=1e-12)
+    assert np.abs(g[8:] - short[8:]).max() > 1e-6
+    eps = 1e-6
+    flat = o.score_global(np.zeros((N, d)), k, 1.0, eps)
+    np.testing.assert_allclose(flat, [_equal_logit_score(t + 1, eps) for t in range(N)], rtol=1e-9)
+
+
 # --------------------------------------------------------------------------- selection
 
 
