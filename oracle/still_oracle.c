@@ -30,7 +30,14 @@
  *     z is a vector of d' entries;
  *   - the gate multiplies N_LA only;
  *   - Top-lambda uses the total order (score descending, index ascending),
- *     NaN ranks lowest, and the result is listed in ascending index order.
+ *     NaN ranks lowest, and the result is listed in ascending index order;
+ *   - salient-cache budget (max_salient > 0; 0 = unbounded, the routing equation
+ *     as written): the paper's long-context experiments cap the number of cached
+ *     salient tokens but the method section gives no rule.  PARITY UNPINNED for the
+ *     choice of rule.  The rule taken here: tokens enter the salient cache in
+ *     routing order; whenever it holds more than max_salient tokens the oldest is
+ *     removed and folded into (s, z) through phi_k exactly like an unselected
+ *     token, so every token outside the local region is counted exactly once.
  *
  * Indices are 0-based here: token i (0-based) is in chunk i / C; the paper's
  * token t is i+1 and its chunk c is i/C + 1.
@@ -301,7 +308,7 @@ static void merge_row(const sa_acc *a, const double *phi_q, const double *S, con
 
 void still_oracle_chunkwise(const double *q, const double *k, const double *v, const double *g,
                             int64_t N, int d, int df, int C, int lam, double sm_scale, double eps,
-                            const double *Wq, const double *bq, const double *Wk, const double *bk,
+                            int64_t max_salient, const double *Wq, const double *bq, const double *Wk, const double *bk,
                             const int32_t *forced_idx, const int64_t *rows, int64_t n_rows,
                             double *y, double *score_out, int32_t *idx_out, double *parts) {
     int64_t T = (N + C - 1) / C;
@@ -326,6 +333,9 @@ void still_oracle_chunkwise(const double *q, const double *k, const double *v, c
     double *phi = (double *)malloc(sizeof(double) * (size_t)dp);
     double *num = (double *)malloc(sizeof(double) * (size_t)d);
     int64_t out_i = 0, row_cursor = 0;
+    /* salient cache of the routed chunks in routing (= position) order; [sal_head, n_sal) is live */
+    int64_t *sal = (int64_t *)malloc(sizeof(int64_t) * (size_t)(N + 1));
+    int64_t n_sal = 0, sal_head = 0;
 
     for (int64_t c = 0; c < T; ++c) {
         /* Linear Attention Branch: the state seen by chunk c holds the LA tokens
@@ -334,6 +344,20 @@ void still_oracle_chunkwise(const double *q, const double *k, const double *v, c
             int64_t b0 = (c - 2) * C;
             for (int64_t i = b0; i < b0 + C; ++i) {
                 if (in_sa[i]) continue;
+                still_oracle_npmap(k + i * d, 1, d, df, Wk, bk, phi);
+                for (int f = 0; f < dp; ++f) {
+                    for (int e = 0; e < d; ++e) S[(size_t)f * d + e] += phi[f] * v[i * d + e];
+                    z[f] += phi[f];
+                }
+            }
+            /* the selected tokens of chunk c-2 enter the salient cache; beyond the budget the oldest
+               leave it for the LA state */
+            for (int j = 0; j < lam; ++j) {
+                int32_t p = idx[(c - 2) * lam + j];
+                if (p >= 0) sal[n_sal++] = p;
+            }
+            while (max_salient > 0 && n_sal - sal_head > max_salient) {
+                int64_t i = sal[sal_head++];
                 still_oracle_npmap(k + i * d, 1, d, df, Wk, bk, phi);
                 for (int f = 0; f < dp; ++f) {
                     for (int e = 0; e < d; ++e) S[(size_t)f * d + e] += phi[f] * v[i * d + e];
@@ -356,12 +380,9 @@ void still_oracle_chunkwise(const double *q, const double *k, const double *v, c
             acc.num = num;
             acc.den = 0.0;
             for (int i = 0; i < d; ++i) num[i] = 0.0;
-            /* q k_SA^T . M_chunk : selected tokens of chunks 0..c-2 */
-            for (int64_t j = 0; j < (c >= 2 ? (c - 1) * lam : 0); ++j) {
-                int32_t p = idx[j];
-                if (p < 0) continue;
-                sa_add(&acc, sm_scale * dotd(q + t * d, k + (int64_t)p * d, d), v + (int64_t)p * d);
-            }
+            /* q k_SA^T . M_chunk : selected tokens of chunks 0..c-2 (those still in the cache) */
+            for (int64_t j = sal_head; j < n_sal; ++j)
+                sa_add(&acc, sm_scale * dotd(q + t * d, k + sal[j] * d, d), v + sal[j] * d);
             /* s_prev : all of chunk c-1 */
             if (c >= 1)
                 for (int64_t p = base - C; p < base; ++p)
@@ -383,6 +404,7 @@ void still_oracle_chunkwise(const double *q, const double *k, const double *v, c
     free(z);
     free(phi);
     free(num);
+    free(sal);
 }
 
 /* ------------------------------------------------------------------------ */
@@ -400,14 +422,14 @@ void still_oracle_chunkwise(const double *q, const double *k, const double *v, c
 
 void still_oracle_recurrent(const double *q, const double *k, const double *v, const double *g,
                             int64_t N, int d, int df, int C, int lam, double sm_scale, double eps,
-                            const double *Wq, const double *bq, const double *Wk, const double *bk,
+                            int64_t max_salient, const double *Wq, const double *bq, const double *Wk, const double *bk,
                             const int32_t *forced_idx, double *y, double *score_out,
                             int32_t *idx_out) {
     int dp = 2 * df;
     int64_t Tn = (N + C - 1) / C;
     double *score = (double *)malloc(sizeof(double) * (size_t)N);
     int64_t *sal = (int64_t *)malloc(sizeof(int64_t) * (size_t)(N + 1));
-    int64_t n_sal = 0;
+    int64_t n_sal = 0, sal_head = 0; /* [sal_head, n_sal) is the live salient cache */
     double *s = (double *)calloc((size_t)dp * d, sizeof(double));
     double *z = (double *)calloc((size_t)dp, sizeof(double));
     double *phi = (double *)malloc(sizeof(double) * (size_t)dp);
@@ -479,6 +501,15 @@ void still_oracle_recurrent(const double *q, const double *k, const double *v, c
                     }
                 }
             }
+            /* budget: the oldest salient pairs leave the cache for the state */
+            while (max_salient > 0 && n_sal - sal_head > max_salient) {
+                int64_t p0 = sal[sal_head++];
+                still_oracle_npmap(k + p0 * d, 1, d, df, Wk, bk, phi);
+                for (int f = 0; f < dp; ++f) {
+                    for (int e = 0; e < d; ++e) s[(size_t)f * d + e] += phi[f] * v[p0 * d + e];
+                    z[f] += phi[f];
+                }
+            }
         }
         /* h_t = local region { max(0, aC) < i <= t } united with the salient pairs. */
         sa_acc acc;
@@ -487,7 +518,7 @@ void still_oracle_recurrent(const double *q, const double *k, const double *v, c
         acc.num = num;
         acc.den = 0.0;
         for (int i = 0; i < d; ++i) num[i] = 0.0;
-        for (int64_t j = 0; j < n_sal; ++j)
+        for (int64_t j = sal_head; j < n_sal; ++j)
             sa_add(&acc, sm_scale * dotd(qt, k + sal[j] * d, d), v + sal[j] * d);
         int64_t lo = (a > 0 ? a * C : 0); /* exclusive, 1-based */
         for (int64_t i = lo + 1; i <= t1; ++i)
@@ -530,7 +561,7 @@ void still_oracle_recurrent(const double *q, const double *k, const double *v, c
 
 int still_oracle_layer(const double *Q, const double *K, const double *V, const double *G, int B,
                        int H, int Hkv, int64_t N, int d, int df, int C, int lam, double sm_scale,
-                       double eps, const double *Wq, const double *bq, const double *Wk,
+                       double eps, int64_t max_salient, const double *Wq, const double *bq, const double *Wk,
                        const double *bk, const int32_t *forced_idx, const int64_t *rows,
                        int64_t n_rows, double *Y, double *score_out, int32_t *idx_out) {
     int64_t T = (N + C - 1) / C;
@@ -547,7 +578,7 @@ int still_oracle_layer(const double *Q, const double *K, const double *V, const 
         const double *k = K + ((size_t)b * Hkv + kv) * N * d;
         const double *v = V + ((size_t)b * Hkv + kv) * N * d;
         still_oracle_chunkwise(q, k, v, G ? G + (size_t)bh * N * d : NULL, N, d, df, C, lam,
-                               sm_scale, eps, Wq + (size_t)h * d * df, bq ? bq + (size_t)h * df : NULL,
+                               sm_scale, eps, max_salient, Wq + (size_t)h * d * df, bq ? bq + (size_t)h * df : NULL,
                                Wk + (size_t)kv * d * df, bk ? bk + (size_t)kv * df : NULL,
                                forced_idx ? forced_idx + (size_t)bh * T * lam : NULL, rows, n_rows,
                                Y + (size_t)bh * n_out * d,

@@ -82,6 +82,7 @@ class HeadParams:
     lam: int
     sm_scale: float
     eps: float = 1e-6
+    max_salient: int = 0  # salient-cache budget per head; 0 = unbounded (rule: oldest out, folded into the LA state)
 
 
 def score_tokenwise(q, k, w, sm_scale, eps=1e-6):
@@ -155,7 +156,7 @@ def chunkwise(q, k, v, Wq, Wk, p: HeadParams, g=None, bq=None, bk=None, forced_i
     parts = np.empty((n_out, 2 * d + 3), dtype=np.float64) if want_parts else None
     _load().still_oracle_chunkwise(
         _d(q), _d(k), _d(v), _d(g), ctypes.c_int64(N), d, df, int(p.C), int(p.lam),
-        ctypes.c_double(p.sm_scale), ctypes.c_double(p.eps), _d(Wq), _d(bq), _d(Wk), _d(bk),
+        ctypes.c_double(p.sm_scale), ctypes.c_double(p.eps), ctypes.c_int64(p.max_salient), _d(Wq), _d(bq), _d(Wk), _d(bk),
         _i32(fi), _i64(rows_a), ctypes.c_int64(n_out if rows_a is not None else 0),
         _d(y), _d(score), _i32(idx) if p.lam > 0 else None, _d(parts),
     )
@@ -179,7 +180,7 @@ def recurrent(q, k, v, Wq, Wk, p: HeadParams, g=None, bq=None, bk=None, forced_i
         fi = np.ascontiguousarray(np.asarray(forced_idx, dtype=np.int32).reshape(T, p.lam))
     _load().still_oracle_recurrent(
         _d(q), _d(k), _d(v), _d(g), ctypes.c_int64(N), d, df, int(p.C), int(p.lam),
-        ctypes.c_double(p.sm_scale), ctypes.c_double(p.eps), _d(Wq), _d(bq), _d(Wk), _d(bk),
+        ctypes.c_double(p.sm_scale), ctypes.c_double(p.eps), ctypes.c_int64(p.max_salient), _d(Wq), _d(bq), _d(Wk), _d(bk),
         _i32(fi), _d(y), _d(score), _i32(idx) if p.lam > 0 else None,
     )
     return {"y": y, "score": score, "idx": idx[:, : p.lam]}
@@ -204,7 +205,7 @@ def layer(Q, K, V, Wq, Wk, p: HeadParams, G=None, bq=None, bk=None, forced_idx=N
         fi = np.ascontiguousarray(np.asarray(forced_idx, dtype=np.int32).reshape(B, H, T, p.lam))
     threads = _load().still_oracle_layer(
         _d(Q), _d(K), _d(V), _d(G), B, H, Hkv, ctypes.c_int64(N), d, df, int(p.C), int(p.lam),
-        ctypes.c_double(p.sm_scale), ctypes.c_double(p.eps), _d(Wq), _d(bq), _d(Wk), _d(bk),
+        ctypes.c_double(p.sm_scale), ctypes.c_double(p.eps), ctypes.c_int64(p.max_salient), _d(Wq), _d(bq), _d(Wk), _d(bk),
         _i32(fi), _i64(rows_a), ctypes.c_int64(n_out if rows_a is not None else 0),
         _d(Y), _d(score), _i32(idx) if p.lam > 0 else None,
     )

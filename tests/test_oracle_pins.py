@@ -288,7 +288,7 @@ def test_lambda_zero_parts_are_local_softmax_and_lagged_linear_attention():
     np.testing.assert_allclose(out["y"], y, rtol=1e-12)
 
 
-def _brute_force(q, k, v, g, Wq, Wk, C, lam, scale, eps):
+def _brute_force(q, k, v, g, Wq, Wk, C, lam, scale, eps, cap=0):
     """The layer from its set definitions, token by token, 1-based as in the paper."""
     N, d = q.shape
     chunk = lambda i: -(-i // C)  # noqa: E731  1-based token -> 1-based chunk
@@ -323,6 +323,8 @@ def _brute_force(q, k, v, g, Wq, Wk, C, lam, scale, eps):
         ct = chunk(t)
         local = {i for i in range(1, t + 1) if chunk(i) >= ct - 1}
         salient = set().union(*[M_SA[c] for c in range(1, ct - 1)]) if ct > 2 else set()
+        if cap > 0:  # budget: of the routed selected tokens only the `cap` most recent stay in the cache
+            salient = set(sorted(salient)[-cap:])
         la = {i for i in range(1, t + 1) if chunk(i) <= ct - 2} - salient
         sets.append((local, salient, la))
         num = np.zeros(d)
@@ -484,3 +486,67 @@ def test_layer_forced_indices_are_taken_per_head():
             one = o.chunkwise(Q[b, h], K[b, 0], V[b, 0], Wq[h], Wk[0], p, forced_idx=forced[b, h])
             np.testing.assert_array_equal(out["y"][b, h], one["y"])
             np.testing.assert_array_equal(out["idx"][b, h], forced[b, h])
+
+
+# --------------------------------------------------------------------------- salient-cache budget
+# The paper caps the salient cache in its long-context experiments without stating a rule; the rule taken
+# (oldest out, folded into the linear state) is this implementation's choice.  These tests pin the
+# implementation to that stated rule, not the rule to the paper.
+
+
+@pytest.mark.parametrize("N,C,lam,cap", [(30, 4, 2, 4), (29, 4, 2, 3), (40, 4, 1, 2), (26, 4, 3, 1), (33, 8, 3, 6)])
+def test_budget_brute_force_tiny(N, C, lam, cap):
+    d, df = 3, 2
+    rng = np.random.default_rng(N * 1000 + C * 100 + lam * 10 + cap)
+    q, k, v = rng.standard_normal((3, N, d))
+    Wq, Wk = rng.standard_normal((2, d, df))
+    g = rng.random((N, d))
+    y, score, idx, sets = _brute_force(q, k, v, g, Wq, Wk, C, lam, 0.7, 1e-6, cap=cap)
+    for local, salient, la in sets:  # still a partition of the prefix, with at most `cap` salient tokens
+        t = max(local)
+        assert local | salient | la == set(range(1, t + 1))
+        assert not (local & salient) and not (local & la) and not (salient & la)
+        assert len(salient) <= cap
+    p = o.HeadParams(C, lam, 0.7, 1e-6, max_salient=cap)
+    for fn in (o.chunkwise, o.recurrent):
+        out = fn(q, k, v, Wq, Wk, p, g=g)
+        np.testing.assert_array_equal(out["idx"], idx)   # the budget does not change which tokens are selected
+        np.testing.assert_allclose(out["y"], y, rtol=1e-9, atol=1e-12)
+
+
+def test_budget_that_is_never_reached_changes_nothing():
+    N, C, lam, d = 96, 8, 3, 5
+    q, k, v, Wq, Wk = _rand_head(N, d)
+    free = o.chunkwise(q, k, v, Wq, Wk, o.HeadParams(C, lam, 0.5))
+    big = o.chunkwise(q, k, v, Wq, Wk, o.HeadParams(C, lam, 0.5, max_salient=(N // C) * lam))
+    np.testing.assert_array_equal(big["y"], free["y"])
+    tight = o.chunkwise(q, k, v, Wq, Wk, o.HeadParams(C, lam, 0.5, max_salient=2 * lam))
+    first_diff = (2 + 2) * C + C   # the third routed chunk pushes the first one out: rows of chunk 4 on
+    np.testing.assert_array_equal(tight["y"][: 4 * C], free["y"][: 4 * C])
+    assert np.abs(tight["y"][4 * C: first_diff] - free["y"][4 * C: first_diff]).max() > 1e-9
+
+
+@pytest.mark.parametrize("N,C,lam,cap", [(100, 16, 4, 8), (128, 16, 16, 32), (77, 8, 2, 5), (90, 8, 8, 8)])
+def test_budget_recurrent_equals_chunkwise(N, C, lam, cap):
+    d = 8
+    q, k, v, Wq, Wk = _rand_head(N, d, scale=1.5)
+    g = RNG.random((N, d))
+    p = o.HeadParams(C, lam, d ** -0.5, max_salient=cap)
+    a = o.chunkwise(q, k, v, Wq, Wk, p, g=g)
+    b = o.recurrent(q, k, v, Wq, Wk, p, g=g)
+    np.testing.assert_allclose(a["y"], b["y"], rtol=1e-9, atol=1e-12)
+
+
+def test_budget_keeps_every_past_token_counted_once():
+    # one-hot values expose each token's weight: positive for every i <= t whether the token is local, cached
+    # or folded into the state after leaving the cache; zero for i > t; the weights of a row sum to one
+    N = d = 32
+    C, lam, cap = 4, 2, 4
+    q, k = RNG.standard_normal((2, N, d)) * 0.3
+    Wq, Wk = RNG.standard_normal((2, d, d)) * 0.3
+    y = o.chunkwise(q, k, np.eye(N), Wq, Wk, o.HeadParams(C, lam, 0.5, max_salient=cap))["y"]
+    for t in range(N):
+        assert np.all(y[t, : t + 1] > 0) and np.all(y[t, t + 1:] == 0)
+    np.testing.assert_allclose(y.sum(1), 1, rtol=1e-12)
+    const = o.chunkwise(q, k, np.full((N, d), 0.25), Wq, Wk, o.HeadParams(C, lam, 0.5, max_salient=cap))["y"]
+    np.testing.assert_allclose(const, 0.25, rtol=1e-12)
