@@ -35,18 +35,22 @@ METRIC = "hybrid-attn prefill tokens/s/layer at Llama-3-8B shape"
 UNIT = "tokens/s"
 
 
-def algorithmic_work(w, lam=None):
-    """FLOPs and bytes the method itself needs for one prefill call (causal-exact pair count)."""
+def algorithmic_work(w, lam=None, max_salient=0):
+    """FLOPs and bytes the method itself needs for one prefill call (causal-exact pair count).  With a
+    salient-cache budget a query of chunk t sees min((t-2) lam, max_salient) cached tokens."""
     lam = w.k if lam is None else lam
     C, d, N = w.C, w.d, w.N
     T = -(-N // C)
     BH, BHkv = w.B * w.H, w.B * w.Hkv
     es = 4 if w.dtype == "fp32" else 2
-    p_sel = C * lam * max(T - 1, 0) * max(T - 2, 0) // 2
+    if max_salient > 0:
+        p_sel = C * sum(min(max(t - 2, 0) * lam, max_salient) for t in range(1, T + 1))
+    else:
+        p_sel = C * lam * max(T - 1, 0) * max(T - 2, 0) // 2
     p_loc = max(T - 1, 0) * C * C + T * C * (C + 1) // 2
     f_sa = 4 * d * (p_sel + p_loc) * BH
     dp = 2 * w.d_f
-    la = lam < C
+    la = lam < C or max_salient > 0
     f_map = 2 * d * w.d_f * N * (BH + BHkv) if la else 0
     f_la = (2 * (C - lam) + 2 * C) * dp * (d + 1) * max(T - 2, 0) * BH if la else 0
     f_score = 2 * d * (2 * C) * C * T * BH  # s_in and s_prev tiles
@@ -318,14 +322,14 @@ def roofline_times(work, peaks):
     return nominal, measured
 
 
-def time_prefill(w, lam, steps, warmup, still, synth, torch, dist, dev, rank, sample_clocks=True):
+def time_prefill(w, lam, steps, warmup, still, synth, torch, dist, dev, rank, sample_clocks=True, max_salient=0):
     """Runs warmup + steps prefill calls of workload w with topk lam on resident inputs.  Every timed step
     has its own CUDA-event pair; the K steps are also bracketed as a whole.  Returns the measurements and
     the tensors (for the end-to-end leg)."""
     wl = w.with_(k=lam, seed=w.seed + 100 * rank)
     Q, K, V = synth.make_qkv(wl, dev)
     Wq, Wk = synth.make_npmap_weights(wl, dev)
-    p = still.StillParams(w.B, w.H, w.Hkv, w.d, w.C, lam, w.torch_dtype)
+    p = still.StillParams(w.B, w.H, w.Hkv, w.d, w.C, lam, w.torch_dtype, max_salient=max_salient)
     Y = torch.empty_like(Q)
     T = -(-w.N // w.C)
     scores = torch.empty(w.B, w.H, w.N, dtype=torch.float32, device=dev)
@@ -358,18 +362,18 @@ def time_prefill(w, lam, steps, warmup, still, synth, torch, dist, dev, rank, sa
             "tensors": (p, Q, K, V, Wq, Wk)}
 
 
-def prefill_companion(name, w, lam, steps, still, synth, torch, dev):
+def prefill_companion(name, w, lam, steps, still, synth, torch, dev, max_salient=0):
     """One more workload in the same run (single GPU): ms per step (median of per-step event pairs), tokens/s
     and the whole-step fraction of the roofline time, with its own clock sample."""
-    m = time_prefill(w, lam, steps, 3, still, synth, torch, None, dev, 0)
+    m = time_prefill(w, lam, steps, 3, still, synth, torch, None, dev, 0, max_salient=max_salient)
     del m["tensors"]
     torch.cuda.empty_cache()
-    work = algorithmic_work(w, lam)
+    work = algorithmic_work(w, lam, max_salient)
     peaks = measured_peaks()
     nominal, measured = roofline_times(work, peaks)
     ms = statistics.median(m["per_step"])
     k_ms = statistics.median(m["kernel_ms"]) if m["kernel_ms"] else None
-    out = {"workload": name, "B": w.B, "H": w.H, "Hkv": w.Hkv, "d": w.d, "N": w.N, "chunk": w.C, "topk": lam,
+    out = {"workload": name, "max_salient": max_salient, "B": w.B, "H": w.H, "Hkv": w.Hkv, "d": w.d, "N": w.N, "chunk": w.C, "topk": lam,
            "steps": steps, "ms_per_step": ms, "tokens_per_s": w.B * w.N / (ms * 1e-3),
            "roofline_frac_nominal": nominal / (ms * 1e-3), "roofline_frac_measured": measured / (ms * 1e-3),
            "workspace_bytes": m["workspace_bytes"], "gpu_launches_per_step": m["launches_per_step"],
@@ -450,8 +454,14 @@ def bench_prefill(args, w, lam, still, synth, torch, dist, dev, rank, world):
             prefill_companion("c2 topk=C/4", W["c2"], 16, 10, still, synth, torch, dev),
             prefill_companion("c4", W["c4"], 128, 2, still, synth, torch, dev),
             prefill_companion("c4 topk=C/4", W["c4"], 32, 2, still, synth, torch, dev),
+            # a capped salient cache (local window 128 + at most 896 cached tokens per head, Sec. 4.3's setting): the
+            # cost per token no longer grows with the sequence -- a quarter of the length takes a quarter of the time
+            prefill_companion("c4 topk=C/4 max_salient=896", W["c4"], 32, 3, still, synth, torch, dev, max_salient=896),
+            prefill_companion("c4 topk=C/4 max_salient=896 N=32768", W["c4"].with_(N=32768), 32, 5, still, synth, torch, dev,
+                              max_salient=896),
             decode_companion("c5", W["c5"], 64, 48, still, synth, torch, dev),
             decode_companion("c5 topk=C/4", W["c5"], 16, 48, still, synth, torch, dev),
+            decode_companion("c5 topk=C/4 max_salient=448", W["c5"], 16, 48, still, synth, torch, dev, max_salient=448),
         ]
 
     cpu = None
@@ -480,22 +490,25 @@ def bench_prefill(args, w, lam, still, synth, torch, dist, dev, rank, world):
     }
 
 
-def decode_bytes(w, lam, t):
+def decode_bytes(w, lam, t, max_salient=0):
     """Bytes a decode step at position t has to move: K and V rows of the routed history that at least one
     query head of the KV group selected (expected size of the union of the group's selections:
     1 - (1 - lam/C)^group of the rows; all rows when lam = C), read once per KV head, plus the two-chunk local
     region and, when the linear branch is in use, its state."""
     rep = w.H // w.Hkv
     union = 1.0 - (1.0 - lam / w.C) ** rep if lam > 0 else 0.0
-    n_hist = max(t // w.C - 1, 0) * w.C * union
+    n_chunks = max(t // w.C - 1, 0)
+    if max_salient > 0 and lam > 0:   # only the last max_salient / lam routed chunks are still cached
+        n_chunks = min(n_chunks, max_salient // lam)
+    n_hist = n_chunks * w.C * union
     return (w.B * w.Hkv * (n_hist + 2 * w.C) * w.d * 2 * 2 +
-            (w.B * w.H * 2 * w.d_f * (w.d + 1) * 4 if lam < w.C else 0))
+            (w.B * w.H * 2 * w.d_f * (w.d + 1) * 4 if (lam < w.C or max_salient > 0) else 0))
 
 
-def time_decode(w, lam, n_steps, warmup, still, synth, torch, dist, dev, rank, reserve=0):
+def time_decode(w, lam, n_steps, warmup, still, synth, torch, dist, dev, rank, reserve=0, max_salient=0):
     """Summarises the prefix into a decode state with the prefill, then times n_steps decode steps (one event
     pair per step and one around all of them)."""
-    p = still.StillParams(w.B, w.H, w.Hkv, w.d, w.C, lam, w.torch_dtype)
+    p = still.StillParams(w.B, w.H, w.Hkv, w.d, w.C, lam, w.torch_dtype, max_salient=max_salient)
     cap = w.N + n_steps + warmup + reserve + 8
     state_bytes = still.state_bytes(p, cap)
     state = torch.zeros(state_bytes, dtype=torch.uint8, device=dev)
@@ -537,14 +550,14 @@ def time_decode(w, lam, n_steps, warmup, still, synth, torch, dist, dev, rank, r
             "state_bytes": state_bytes, "t": t, "ctx": (p, state, cap, ins, y, Wq, Wk, wl)}
 
 
-def decode_companion(name, w, lam, n_steps, still, synth, torch, dev):
-    m = time_decode(w, lam, n_steps, 3, still, synth, torch, None, dev, 0)
+def decode_companion(name, w, lam, n_steps, still, synth, torch, dev, max_salient=0):
+    m = time_decode(w, lam, n_steps, 3, still, synth, torch, None, dev, 0, max_salient=max_salient)
     del m["ctx"]
     torch.cuda.empty_cache()
     peaks = measured_peaks()
     ms = statistics.median(m["per_step"])
-    by = decode_bytes(w, lam, m["t"])
-    return {"workload": name, "B": w.B, "H": w.H, "Hkv": w.Hkv, "d": w.d, "prefix": w.N, "chunk": w.C, "topk": lam,
+    by = decode_bytes(w, lam, m["t"], max_salient)
+    return {"workload": name, "max_salient": max_salient, "B": w.B, "H": w.H, "Hkv": w.Hkv, "d": w.d, "prefix": w.N, "chunk": w.C, "topk": lam,
             "steps": n_steps, "ms_per_step": ms, "ms_per_step_max": max(m["per_step"]),
             "tokens_per_s": w.B / (ms * 1e-3), "algorithmic_bytes_per_step": by,
             "roofline_frac_nominal": (by / 8e12) / (ms * 1e-3),

@@ -89,9 +89,21 @@ typedef struct still_params {
     float sm_scale;     /* multiplies q.k in the score and in the SA branch (1 = the main     */
                         /* text's exp(qk^T); d^-1/2 = App. A.1, Eq. softmax_attention)       */
     float eps;          /* epsilon of the Self-Saliency Score                                */
-    int64_t max_salient;/* reserved, must be 0: the salient cache is unbounded (Eq.          */
-                        /* cache_routing_sum as written)                                      */
+    int64_t max_salient;/* budget of the salient cache per query head, in tokens; 0 = unbounded */
+                        /* (Eq. cache_routing_sum as written).  See below.                   */
 } still_params_t;
+
+/*
+ * Salient-cache budget.  The paper's long-context experiments (Sec. 4.3) cap the number of cached salient
+ * tokens, but its method section states no rule for what happens at the cap; the rule below is this
+ * library's choice.  Selected tokens enter a head's salient cache in routing order, a chunk's top-k at a time;
+ * when the cache would exceed max_salient tokens the oldest leave it and are folded into the linear state
+ * (s, z) through phi_k, exactly as an unselected token is.  Every token outside the two-chunk local region is
+ * thus counted once, in the softmax branch or in the linear branch, and the cost per token no longer grows
+ * with the sequence (Eq. complexity's O(N) with a constant cache).  Selection itself is unchanged.
+ * Supported: max_salient a positive multiple of topk (whole chunks' selections leave together), bf16 inputs
+ * on the tensor-core kernels (chunk 64 or 128, d_f >= 64); otherwise STILL_ERR_UNSUPPORTED.
+ */
 
 /* Bytes of workspace still_hybrid_attn_fwd needs for a sequence of N tokens
  * (0 if the parameters are invalid).  Host-only arithmetic, no CUDA call. */
@@ -109,9 +121,13 @@ size_t still_state_bytes(const still_params_t *p, int64_t max_tokens);
  *   header   : 256 bytes, int32 words {magic, version, B, H, Hkv, d, d_f, chunk,
  *              topk, dtype, capacity_lo, capacity_hi, t_lo, t_hi, status, 0...};
  *              t = tokens consumed so far.
- *   k_cache, v_cache : [B, Hkv, capacity, d] in dtype -- the K/V history
+ *   k_cache, v_cache : [B, Hkv, rows, d] in dtype -- the K/V history
  *              (local region + every earlier token; the salient pairs of Eq.
- *              cache_routing_sum are rows of it named by sel_idx).
+ *              cache_routing_sum are rows of it named by sel_idx).  rows = capacity,
+ *              position q in row q.  With a salient-cache budget the store is a ring
+ *              of rows = min(capacity, (max_salient / topk + 3) * chunk) -- the cached
+ *              chunks, the two-chunk local region and the chunk being routed --
+ *              with position q in row q % rows: it does not grow with the sequence.
  *   score    : [B, H, capacity] fp32 -- Self-Saliency Score of every token.
  *   sel_idx  : [B, H, capacity / chunk, topk] int32 -- salient positions of each
  *              routed chunk, ascending, -1 padded (rows of chunks not yet routed

@@ -53,12 +53,13 @@ class StillParams:
     d_f: int | None = None
     sm_scale: float | None = None
     eps: float = 1e-6
+    max_salient: int = 0  # salient-cache budget per query head (a multiple of topk); 0 = unbounded
 
     def c(self) -> _CParams:
         return _CParams(
             self.B, self.H, self.Hkv, self.d, self.d if self.d_f is None else self.d_f, self.chunk, self.topk,
             DTYPE_FP32 if self.dtype == torch.float32 else DTYPE_BF16,
-            float(self.d) ** -0.5 if self.sm_scale is None else self.sm_scale, self.eps, 0,
+            float(self.d) ** -0.5 if self.sm_scale is None else self.sm_scale, self.eps, self.max_salient,
         )
 
 

@@ -39,16 +39,22 @@ static int validate(const still_params_t *p) {
     if (p->B <= 0 || p->H <= 0 || p->Hkv <= 0 || p->H % p->Hkv != 0) return STILL_ERR_INVALID_ARG;
     if (p->topk < 0 || p->topk > p->chunk) return STILL_ERR_INVALID_ARG;
     if (!(p->sm_scale > 0.f) || !(p->eps > 0.f)) return STILL_ERR_INVALID_ARG;
-    if (p->max_salient != 0) return STILL_ERR_UNSUPPORTED;
+    if (p->max_salient < 0) return STILL_ERR_INVALID_ARG;
     if (p->dtype != STILL_DTYPE_FP32 && p->dtype != STILL_DTYPE_BF16) return STILL_ERR_UNSUPPORTED;
     if (p->d != 64 && p->d != 128) return STILL_ERR_UNSUPPORTED;
     if (p->chunk != 32 && p->chunk != 64 && p->chunk != 128) return STILL_ERR_UNSUPPORTED;
     if (p->d_f != 32 && p->d_f != 64 && p->d_f != 128) return STILL_ERR_UNSUPPORTED;
     if (p->d_f > p->d) return STILL_ERR_UNSUPPORTED;
+    if (p->max_salient > 0) {
+        // budget of the salient cache: whole chunks' worth of selections, on the tensor-core kernels
+        if (p->topk == 0 || p->max_salient % p->topk != 0 || p->max_salient / p->topk > (1 << 20)) return STILL_ERR_UNSUPPORTED;
+        if (!tc_supported(p) || !tc_la_supported(p)) return STILL_ERR_UNSUPPORTED;
+    }
     return STILL_OK;
 }
 
-static inline bool la_active(const still_params_t *p) { return p->topk < p->chunk; }
+// The linear branch runs when a chunk can have unselected tokens, or when cached tokens can leave the cache.
+static inline bool la_active(const still_params_t *p) { return p->topk < p->chunk || p->max_salient > 0; }
 
 // Workspace plan of the prefill.
 struct FwdPlan {
@@ -117,8 +123,9 @@ static int plan_state(const still_params_t *p, long long max_tokens, still_state
     };
     L->capacity = cap;
     L->header = take(256);
-    L->k_cache = take(BHkv * (size_t)cap * p->d * es);
-    L->v_cache = take(BHkv * (size_t)cap * p->d * es);
+    const size_t kvr = (size_t)state_kv_rows(p, cap);
+    L->k_cache = take(BHkv * kvr * p->d * es);
+    L->v_cache = take(BHkv * kvr * p->d * es);
     L->score = take(BH * (size_t)cap * 4);
     L->sel_idx = take(BH * (size_t)(cap / p->chunk) * (size_t)std::max(p->topk, 1) * 4);
     L->sel_mask = take(BH * (size_t)(cap / p->chunk) * (size_t)(p->chunk / 32) * 4);
@@ -337,12 +344,18 @@ static int fwd_typed(const still_params_t *p, long long N, const T *Q, const T *
     if (state) {
         const size_t es = sizeof(T);
         const size_t BH = (size_t)p->B * p->H, BHkv = (size_t)p->B * p->Hkv;
-        STILL_CUDA(cudaMemcpy2DAsync(state + L.k_cache, (size_t)L.capacity * p->d * es, K,
-                                     (size_t)N * p->d * es, (size_t)N * p->d * es, BHkv,
-                                     cudaMemcpyDeviceToDevice, st));
-        STILL_CUDA(cudaMemcpy2DAsync(state + L.v_cache, (size_t)L.capacity * p->d * es, V,
-                                     (size_t)N * p->d * es, (size_t)N * p->d * es, BHkv,
-                                     cudaMemcpyDeviceToDevice, st));
+        // K / V history: the whole sequence, or with a budget the last kvr positions into their ring rows
+        // (position q in row q % kvr: at most two contiguous runs)
+        const long long kvr = state_kv_rows(p, L.capacity), first = std::max<long long>(0, N - kvr);
+        const size_t row = (size_t)p->d * es;
+        for (long long q0 = first; q0 < N;) {
+            const long long r0 = q0 % kvr, run = std::min<long long>(N - q0, kvr - r0);
+            STILL_CUDA(cudaMemcpy2DAsync(state + L.k_cache + r0 * row, kvr * row, reinterpret_cast<const char *>(K) + q0 * row,
+                                         (size_t)N * row, run * row, BHkv, cudaMemcpyDeviceToDevice, st));
+            STILL_CUDA(cudaMemcpy2DAsync(state + L.v_cache + r0 * row, kvr * row, reinterpret_cast<const char *>(V) + q0 * row,
+                                         (size_t)N * row, run * row, BHkv, cudaMemcpyDeviceToDevice, st));
+            q0 += run;
+        }
         STILL_CUDA(cudaMemcpy2DAsync(state + L.score, (size_t)L.capacity * 4, sc, (size_t)N * 4,
                                      (size_t)N * 4, BH, cudaMemcpyDeviceToDevice, st));
         if (p->topk > 0)

@@ -285,16 +285,28 @@ npmap_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
 // Normaliser prefix z (Eq. cache_routing_sum): z after chunk c = sum over the chunks 0..c of the features
 // of their unselected tokens = (column sums of phi(K) over the chunk) - (rows of its selected tokens).
 // ------------------------------------------------------------------------------------------
-// grid (routed chunks, B*H), 2 d_f threads: zpre[bh][c][f] = csum[kv][c][f] - sum_i phi(K)[sel[bh][c][i]][f]
+// grid (routed chunks, B*H), 2 d_f threads: zpre[bh][c][f] = csum[kv][c][f] - sum_i phi(K)[sel[bh][c][i]][f], plus,
+// with a salient-cache budget of `window` chunks, the selected rows of chunk c - window, which leave the cache
+// for the state when chunk c is routed.
 __global__ void z_delta_kernel(const float *__restrict__ csum, const __nv_bfloat16 *__restrict__ phiK,
                                const int32_t *__restrict__ sel_idx, float *__restrict__ zpre, int H, int Hkv, long long N,
-                               int Tn, int n_routed, int lam, int NF) {
+                               int Tn, int n_routed, int lam, int C, int window, int NF) {
     const int c = blockIdx.x, bh = blockIdx.y, b = bh / H, h = bh % H, kv = b * Hkv + h / (H / Hkv), f = threadIdx.x;
-    float d = csum[((long long)kv * Tn + c) * NF + f];
-    const int32_t *si = sel_idx + ((long long)bh * Tn + c) * lam;
-    for (int i = 0; i < lam; ++i) {
-        const int p = si[i];
-        if (p >= 0) d -= __bfloat162float(phiK[((long long)kv * N + p) * NF + f]);
+    float d = 0.f;
+    if (lam < C) {   // (with lam = C every token of the chunk is selected: nothing is left over)
+        d = csum[((long long)kv * Tn + c) * NF + f];
+        const int32_t *si = sel_idx + ((long long)bh * Tn + c) * lam;
+        for (int i = 0; i < lam; ++i) {
+            const int p = si[i];
+            if (p >= 0) d -= __bfloat162float(phiK[((long long)kv * N + p) * NF + f]);
+        }
+    }
+    if (window > 0 && c >= window) {
+        const int32_t *si = sel_idx + ((long long)bh * Tn + (c - window)) * lam;
+        for (int i = 0; i < lam; ++i) {
+            const int p = si[i];
+            if (p >= 0) d += __bfloat162float(phiK[((long long)kv * N + p) * NF + f]);
+        }
     }
     zpre[((long long)bh * n_routed + c) * NF + f] = d;
 }
@@ -352,7 +364,8 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 const __nv_bfloat16 *__restrict__ bq, const __nv_bfloat16 *__restrict__ G,
                 const int32_t *__restrict__ sel_idx, const float *__restrict__ zpre, __nv_bfloat16 *__restrict__ y_part,
                 float *__restrict__ d_part, float *__restrict__ S_out, float *__restrict__ seg_sums, int *status, int H, int Hkv,
-                int N, int C, int lam, long long part_stride_y, long long part_stride_d, int seg_chunks, int n_seg, int sums_only) {
+                int N, int C, int lam, int window, long long part_stride_y, long long part_stride_d, int seg_chunks, int n_seg,
+                int sums_only) {
     using P = FusedPlan<D, DF>;
     constexpr int NF = 2 * DF;
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -379,8 +392,12 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const int NU = (!sums_only && seg == n_seg - 1) ? NU_all : min(NU_all, (seg + 1) * seg_chunks * sc);
     const int b_first = u_first / 2;            // blocks of 128 query rows: [b_first, NB)
     const int NB = sums_only ? b_first : (NU + 1) / 2;
-    const int nu0 = (u_first / sc - 2) * sc;    // first update tile of the segment (64-token sub-chunks of routed chunks)
-    const int n_upd = NU > u_first ? ((NU - 1) / sc - 1) * sc - nu0 : 0;
+    // Update tiles: per routed chunk its sc sub-chunks (selected rows zeroed) and, with a salient-cache budget of
+    // `window` chunks, the sc sub-chunks of the chunk `window` back with everything but its selected rows zeroed:
+    // those tokens leave the cache for the state when the chunk is routed.
+    const int per_chunk = window > 0 ? 2 * sc : sc;
+    const int nu0 = (u_first / sc - 2) * per_chunk;    // first update tile of the segment
+    const int n_upd = NU > u_first ? ((NU - 1) / sc - 1) * per_chunk - nu0 : 0;
     const bool has_init = !sums_only && seg > 0;
     __nv_bfloat16 *y_out = y_part + (long long)half * part_stride_y;
     float *d_out = d_part + (long long)half * part_stride_d;
@@ -451,11 +468,16 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 }
                 if (nu < n_upd && mbar_try_wait(u_empty + (nu & 1), ((nu >> 1) & 1) ^ 1)) {
                     uint8_t *stg = smem + P::oU + (nu & 1) * P::kUStage;
+                    // tile a = nu0 + nu: chunk a / per_chunk, then which of its tiles; a leaving-tile reads the chunk
+                    // `window` back (before there is one, any valid tile: all its rows are zeroed)
+                    const int a_t = nu0 + nu, cc = a_t / per_chunk, rt = a_t % per_chunk;
+                    const int src = (rt >= sc && cc >= window) ? cc - window : cc;
+                    const int tile_sub = src * sc + rt % sc;
                     mbar_expect_tx(u_full + (nu & 1), P::kUStage);
                     for (int a = 0; a < DF / 64; ++a)  // phi(K) half: MN-major, 64-feature atoms 64 rows apart
-                        tma_load_2d(stg + a * (64 * 128), &tm_phik, u_full + (nu & 1), half * DF + a * 64, kv_row0 + (nu0 + nu) * 64);
+                        tma_load_2d(stg + a * (64 * 128), &tm_phik, u_full + (nu & 1), half * DF + a * 64, kv_row0 + tile_sub * 64);
                     for (int a = 0; a < D / 64; ++a)   // V: M-major A operand, 64-column atoms 64 rows apart
-                        tma_load_2d(stg + P::kPhiK + a * (64 * 128), &tm_v, u_full + (nu & 1), a * 64, kv_row0 + (nu0 + nu) * 64);
+                        tma_load_2d(stg + P::kPhiK + a * (64 * 128), &tm_v, u_full + (nu & 1), a * 64, kv_row0 + tile_sub * 64);
                     ++nu;
                     progressed = true;
                 }
@@ -529,7 +551,7 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             for (int u = u_first; u < NU && ok && !sums_only; ++u) {
                 if (u % sc == 0) {
                     // the chunk that has just left the local region: sub-chunks of chunk u / sc - 2
-                    for (int j = 0; j < sc && ok; ++j) ok = issue_update();
+                    for (int j = 0; j < per_chunk && ok; ++j) ok = issue_update();
                     if (!ok) break;
                 }
                 ok = mbar_wait(pq_full + (u & 1), (nq >> 1) & 1, abort_flag, status, 65);
@@ -561,26 +583,39 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         // state.  The chunk's indices are fetched before the tile is waited for.
         bool ok = true;
         for (int nu = 0; nu < n_upd; ++nu) {
-            const int chunk = (nu0 + nu) / sc, sub = (nu0 + nu) % sc;
-            const int32_t *si = sel_idx + ((long long)bh * Tn + chunk) * lam;
+            const int a_t = nu0 + nu, cc = a_t / per_chunk, rt = a_t % per_chunk, sub = rt % sc;
+            const bool leaving = rt >= sc;                       // tile of the tokens that leave the salient cache
+            const int chunk = leaving ? cc - window : cc;        // (chunk < 0: nothing leaves yet, every row is zeroed)
             int row[4];
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
                 const int i = lane + 32 * q;
-                row[q] = i < lam ? si[i] - (chunk * C + sub * 64) : -1;   // row within this 64-token tile
+                row[q] = (i < lam && chunk >= 0) ? sel_idx[((long long)bh * Tn + chunk) * lam + i] - (chunk * C + sub * 64) : -1;
             }
+            // the selected rows of the tile as a 64-bit set
+            uint32_t lo = 0u, hi = 0u;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                if (row[q] >= 0 && row[q] < 32) lo |= 1u << row[q];
+                if (row[q] >= 32 && row[q] < 64) hi |= 1u << (row[q] - 32);
+            }
+            lo = __reduce_or_sync(0xffffffffu, lo);
+            hi = __reduce_or_sync(0xffffffffu, hi);
+            if (leaving) { lo = ~lo; hi = ~hi; }                 // rows to zero: the selected ones, or all the others
             if (ok) ok = mbar_wait(u_full + (nu & 1), (nu >> 1) & 1, abort_flag, status, 67);
             ok = __all_sync(0xffffffffu, ok);
             if (ok) {
                 uint8_t *tile = smem + P::oU + (nu & 1) * P::kUStage;
 #pragma unroll
-                for (int q = 0; q < 4; ++q)
-                    if (row[q] >= 0 && row[q] < 64) {
+                for (int hh = 0; hh < 2; ++hh) {                 // lane l looks after rows l and l + 32
+                    if (((hh == 0 ? lo : hi) >> lane) & 1u) {
+                        const int rz = hh * 32 + lane;
 #pragma unroll
                         for (int piece = 0; piece < DF / 8; ++piece)   // 16-byte pieces of the token's feature half
-                            *reinterpret_cast<uint4 *>(tile + (piece >> 3) * (64 * 128) + row[q] * 128 + ((piece & 7) << 4)) =
+                            *reinterpret_cast<uint4 *>(tile + (piece >> 3) * (64 * 128) + rz * 128 + ((piece & 7) << 4)) =
                                 make_uint4(0, 0, 0, 0);
                     }
+                }
                 fence_proxy_async();
             }
             __syncwarp();
@@ -879,7 +914,8 @@ int launch_fused(const still_params_t *p, long long N, const void *Q, const void
         dim3 grid((unsigned)BH, 2, (unsigned)(pass == 0 ? n_seg - 1 : n_seg));   // head, feature half, segment
         la_fused_kernel<D, DF><<<grid, 384, Plan::kTotal, st>>>(tq, tw, tk, tv, (const bf *)bq, (const bf *)G, sel_idx, zpre,
                                                                (bf *)y_part, d_part, S_out, seg_sums, status, p->H, p->Hkv, (int)N,
-                                                               p->chunk, p->topk, (long long)BH * N * D, (long long)BH * N,
+                                                               p->chunk, p->topk, p->topk > 0 ? (int)(p->max_salient / p->topk) : 0,
+                                                               (long long)BH * N * D, (long long)BH * N,
                                                                seg_chunks, n_seg, pass == 0 ? 1 : 0);
         ++*launches;
         if (cudaGetLastError() != cudaSuccess) return STILL_ERR_CUDA;
@@ -927,7 +963,8 @@ int tc_la_branch(const still_params_t *p, long long N, const void *Q, const void
     // z after every routed chunk (per query head: the selection is per query head)
     if (n_routed > 0) {
         z_delta_kernel<<<dim3((unsigned)n_routed, (unsigned)BH), NF, 0, st>>>(csum, (const bf *)phiK, sel_idx, zpre, p->H, p->Hkv,
-                                                                                N, (int)Tn, n_routed, p->topk, NF);
+                                                                                N, (int)Tn, n_routed, p->topk, C,
+                                                                                p->topk > 0 ? (int)(p->max_salient / p->topk) : 0, NF);
         ++*launches;
         if (cudaGetLastError() != cudaSuccess) return STILL_ERR_CUDA;
     }

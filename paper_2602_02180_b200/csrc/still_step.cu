@@ -22,6 +22,12 @@ namespace still {
 
 constexpr int kMaxSplits = 32;  // history splits; one more partial holds the local region
 
+long long state_kv_rows(const still_params_t *p, long long capacity) {
+    if (p->max_salient <= 0 || p->topk <= 0) return capacity;
+    const long long window = p->max_salient / p->topk;   // chunks whose selections stay cached
+    return std::min<long long>(capacity, (window + 3) * p->chunk);
+}
+
 size_t step_scratch_bytes(const still_params_t *p, long long) {
     return (size_t)p->B * p->H * (kMaxSplits + 1) * (p->d + 2) * sizeof(float);
 }
@@ -80,7 +86,7 @@ __global__ void step_append_score_kernel(T *__restrict__ kc, T *__restrict__ vc,
                                          float *__restrict__ score, int32_t *__restrict__ hdr,
                                          const T *__restrict__ q, const T *__restrict__ k,
                                          const T *__restrict__ v, StateKey key, int H, int Hkv, long long cap,
-                                         int d, int C, long long t, float scale, float eps) {
+                                         long long kvr, int d, int C, long long t, float scale, float eps) {
     __shared__ float qs[128];
     const int h = blockIdx.x, b = blockIdx.y, rep = H / Hkv, kv = h / rep, lane = threadIdx.x;
     {
@@ -91,10 +97,11 @@ __global__ void step_append_score_kernel(T *__restrict__ kc, T *__restrict__ vc,
         }
     }
     const T *kn = k + ((long long)b * Hkv + kv) * d;
-    T *krow = kc + (((long long)b * Hkv + kv) * cap + t) * d;
+    // K / V rows live in a ring of kvr rows per KV head (kvr = capacity unless the salient cache has a budget)
+    T *krow = kc + (((long long)b * Hkv + kv) * kvr + t % kvr) * d;
     if (h % rep == 0) {
         const T *vn = v + ((long long)b * Hkv + kv) * d;
-        T *vrow = vc + (((long long)b * Hkv + kv) * cap + t) * d;
+        T *vrow = vc + (((long long)b * Hkv + kv) * kvr + t % kvr) * d;
         for (int i = lane; i < d; i += 32) {
             krow[i] = kn[i];
             vrow[i] = vn[i];
@@ -112,7 +119,7 @@ __global__ void step_append_score_kernel(T *__restrict__ kc, T *__restrict__ vc,
             long long pos = t - (C - 1) + j;
             if (pos >= 0) {
                 // the new key is read from the input, not from the cache row another block writes
-                const T *kr = (pos == t) ? kn : kc + (((long long)b * Hkv + kv) * cap + pos) * d;
+                const T *kr = (pos == t) ? kn : kc + (((long long)b * Hkv + kv) * kvr + pos % kvr) * d;
                 float acc = 0.f;
                 for (int x = 0; x < d; ++x) acc = fmaf(qs[x], ld_f(kr + x), acc);
                 l[i] = acc * scale;
@@ -123,13 +130,15 @@ __global__ void step_append_score_kernel(T *__restrict__ kc, T *__restrict__ vc,
     if (lane == 0) score[((long long)b * H + h) * cap + t] = s;
 }
 
-// grid (H, B), 256 threads.  Routes chunk cr (complete, C tokens).
+// grid (H, B), 256 threads.  Routes chunk cr (complete, C tokens): top-k into sel_idx / sel_mask, the other tokens
+// into (S, z).  With a salient-cache budget of `window` chunks the selected tokens of chunk cr - window leave the
+// cache at the same moment and are folded into (S, z) as well.
 template <typename T>
 __global__ void __launch_bounds__(256)
 step_route_kernel(const T *__restrict__ kc, const T *__restrict__ vc, const float *__restrict__ score,
                   int32_t *__restrict__ sel_idx, uint32_t *__restrict__ sel_mask, float *__restrict__ S,
                   float *__restrict__ z, const T *__restrict__ Wk, const T *__restrict__ bk, const int32_t *__restrict__ hdr,
-                  int H, int Hkv, long long cap, int d, int df, int C, int lam, long long cr) {
+                  int H, int Hkv, long long cap, long long kvr, int d, int df, int C, int lam, long long cr, int window) {
     extern __shared__ float smem[];
     if (hdr[14] != 0) return;   // the step's first kernel found the state not to match the call
     const int dp = 2 * df;
@@ -139,59 +148,70 @@ step_route_kernel(const T *__restrict__ kc, const T *__restrict__ vc, const floa
     float *sc = xs + 8 * d;           // [C]
     int *flag = reinterpret_cast<int *>(sc + C);  // [C]
     const int h = blockIdx.x, b = blockIdx.y, kv = h / (H / Hkv);
-    const long long bh = (long long)b * H + h, base = cr * C;
+    const long long bh = (long long)b * H + h;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (int i = threadIdx.x; i < C; i += blockDim.x) {
-        sc[i] = score[bh * cap + base + i];
+        sc[i] = score[bh * cap + cr * C + i];
         flag[i] = 0;
     }
     __syncthreads();
-    if (lam > 0) select_chunk(sc, flag, C, C, lam, base, sel_idx + (bh * (cap / C) + cr) * lam);
+    if (lam > 0) select_chunk(sc, flag, C, C, lam, cr * C, sel_idx + (bh * (cap / C) + cr) * lam);
     __syncthreads();
     if (threadIdx.x < C / 32) {  // the same selection as bit masks (read by the split-KV pass)
         uint32_t bits = 0u;
         for (int j = 0; j < 32; ++j) bits |= (flag[threadIdx.x * 32 + j] ? 1u : 0u) << j;
         sel_mask[(bh * (cap / C) + cr) * (C / 32) + threadIdx.x] = bits;
     }
-    if (lam >= C) return;  // nothing goes to the linear branch
-    const T *kh = kc + (((long long)b * Hkv + kv) * cap + base) * d;
-    const T *vh = vc + (((long long)b * Hkv + kv) * cap + base) * d;
-    for (int i = threadIdx.x; i < C * d; i += blockDim.x) vs[i] = ld_f(vh + i);
     const T *Wh = Wk + (long long)kv * d * df;
     const T *bh_ = bk ? bk + (long long)kv * df : nullptr;
-    float *xw = xs + warp * d;
-    for (int r = warp; r < C; r += 8) {
-        float ep[4], en[4];
-        if (!flag[r]) {
-            for (int i = lane; i < d; i += 32) xw[i] = ld_f(kh + (long long)r * d + i);
-            __syncwarp();
-            npmap_row(xw, Wh, bh_, d, df, lane, ep, en);
-        }
-#pragma unroll
-        for (int jj = 0; jj < 4; ++jj)
-            if (jj < (df >> 5)) {
-                int j = lane + 32 * jj;
-                // features are rounded to the storage type, as the prefill stores them
-                T a, c2;
-                st_f(&a, flag[r] ? 0.f : ep[jj]);
-                st_f(&c2, flag[r] ? 0.f : en[jj]);
-                ph[r * dp + j] = ld_f(&a);
-                ph[r * dp + df + j] = ld_f(&c2);
-            }
-        __syncwarp();
-    }
-    __syncthreads();
     float *Sh = S + bh * dp * d;
-    for (int idx = threadIdx.x; idx < dp * d; idx += blockDim.x) {
-        int f = idx / d, e = idx - f * d;
-        float acc = Sh[idx];
-        for (int i = 0; i < C; ++i) acc = fmaf(ph[i * dp + f], vs[i * d + e], acc);
-        Sh[idx] = acc;
-    }
-    for (int f = threadIdx.x; f < dp; f += blockDim.x) {
-        float acc = z[bh * dp + f];
-        for (int i = 0; i < C; ++i) acc += ph[i * dp + f];
-        z[bh * dp + f] = acc;
+    // pass 0: the unselected tokens of chunk cr; pass 1: the selected tokens of the chunk that leaves the cache
+    for (int pass = 0; pass < 2; ++pass) {
+        const long long chunk = pass == 0 ? cr : cr - window;
+        if (pass == 0 ? lam >= C : (window <= 0 || chunk < 0)) continue;   // nothing to fold in this pass
+        __syncthreads();
+        if (pass == 1) {   // fold[r] = 1 for the tokens to fold: here the chunk's selected ones, recorded when it was routed
+            for (int i = threadIdx.x; i < C; i += blockDim.x)
+                flag[i] = !((sel_mask[(bh * (cap / C) + chunk) * (C / 32) + i / 32] >> (i & 31)) & 1u);
+            __syncthreads();
+        }
+        const long long base = chunk * C;
+        const T *kh = kc + (((long long)b * Hkv + kv) * kvr + base % kvr) * d;   // (a chunk never straddles the ring's end)
+        const T *vh = vc + (((long long)b * Hkv + kv) * kvr + base % kvr) * d;
+        for (int i = threadIdx.x; i < C * d; i += blockDim.x) vs[i] = ld_f(vh + i);
+        float *xw = xs + warp * d;
+        for (int r = warp; r < C; r += 8) {   // flag[r] != 0: the token stays out of this pass
+            float ep[4], en[4];
+            if (!flag[r]) {
+                for (int i = lane; i < d; i += 32) xw[i] = ld_f(kh + (long long)r * d + i);
+                __syncwarp();
+                npmap_row(xw, Wh, bh_, d, df, lane, ep, en);
+            }
+#pragma unroll
+            for (int jj = 0; jj < 4; ++jj)
+                if (jj < (df >> 5)) {
+                    int j = lane + 32 * jj;
+                    // features are rounded to the storage type, as the prefill stores them
+                    T a, c2;
+                    st_f(&a, flag[r] ? 0.f : ep[jj]);
+                    st_f(&c2, flag[r] ? 0.f : en[jj]);
+                    ph[r * dp + j] = ld_f(&a);
+                    ph[r * dp + df + j] = ld_f(&c2);
+                }
+            __syncwarp();
+        }
+        __syncthreads();
+        for (int idx = threadIdx.x; idx < dp * d; idx += blockDim.x) {
+            int f = idx / d, e = idx - f * d;
+            float acc = Sh[idx];
+            for (int i = 0; i < C; ++i) acc = fmaf(ph[i * dp + f], vs[i * d + e], acc);
+            Sh[idx] = acc;
+        }
+        for (int f = threadIdx.x; f < dp; f += blockDim.x) {
+            float acc = z[bh * dp + f];
+            for (int i = 0; i < C; ++i) acc += ph[i * dp + f];
+            z[bh * dp + f] = acc;
+        }
     }
 }
 
@@ -361,7 +381,7 @@ static int step_typed(const still_params_t *p, char *state, const still_state_la
                       const T *q, const T *k, const T *v, const T *g, const T *Wq, const T *bq,
                       const T *Wk, const T *bk, T *y, cudaStream_t st, int *launches) {
     const int C = p->chunk, d = p->d, df = p->d_f, lam = p->topk;
-    const long long cap = L->capacity;
+    const long long cap = L->capacity, kvr = state_kv_rows(p, cap);
     T *kc = reinterpret_cast<T *>(state + L->k_cache), *vc = reinterpret_cast<T *>(state + L->v_cache);
     float *score = reinterpret_cast<float *>(state + L->score);
     int32_t *sel = reinterpret_cast<int32_t *>(state + L->sel_idx);
@@ -369,11 +389,12 @@ static int step_typed(const still_params_t *p, char *state, const still_state_la
     float *S = reinterpret_cast<float *>(state + L->S), *z = reinterpret_cast<float *>(state + L->z);
     float *part = reinterpret_cast<float *>(state + L->scratch);
     int32_t *hdr = reinterpret_cast<int32_t *>(state + L->header);
-    const bool la = lam < C;
+    const int window = lam > 0 ? (int)(p->max_salient / lam) : 0;   // chunks whose selections the salient cache holds
+    const bool la = lam < C || window > 0;
 
     const StateKey key{p->B, p->H, p->Hkv, p->d, p->d_f, p->chunk, p->topk, p->dtype, cap, t};
     step_append_score_kernel<T><<<dim3(p->H, p->B), 32, 0, st>>>(kc, vc, score, hdr, q, k, v, key, p->H, p->Hkv,
-                                                                  cap, d, C, t, p->sm_scale, p->eps);
+                                                                  cap, kvr, d, C, t, p->sm_scale, p->eps);
     ++*launches;
     STILL_CUDA(cudaGetLastError());
 
@@ -383,7 +404,7 @@ static int step_typed(const still_params_t *p, char *state, const still_state_la
         STILL_CUDA(cudaFuncSetAttribute(step_route_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)smem));
         step_route_kernel<T><<<dim3(p->H, p->B), 256, smem, st>>>(kc, vc, score, sel, smask, S, z, Wk, bk, hdr, p->H,
-                                                                  p->Hkv, cap, d, df, C, lam, c_cur - 2);
+                                                                  p->Hkv, cap, kvr, d, df, C, lam, c_cur - 2, window);
         ++*launches;
         STILL_CUDA(cudaGetLastError());
     }
@@ -393,7 +414,9 @@ static int step_typed(const still_params_t *p, char *state, const still_state_la
     if constexpr (sizeof(T) == 2) {
         // bf16: tensor-core split-KV pass, the query heads of a KV group share every K / V row read
         if (p->H / p->Hkv > 16) return STILL_ERR_UNSUPPORTED;  // the group's heads are the 16 rows of one MMA tile
-        const long long nb = (t + 32) / 32;  // 32-position key blocks
+        // with a budget, the routed chunks still cached are the last `window` ones before the local region
+        const long long first_pos = window > 0 ? std::max<long long>(0, c_cur - 1 - window) * C : 0;
+        const long long nb = (t + 32) / 32 - first_pos / 32;  // 32-position key blocks
         const long long groups = (long long)p->B * p->Hkv;
         const long long want = (6 * 148 + groups - 1) / groups;  // about six waves of CTAs
         n_splits = (int)std::max<long long>(1, std::min<long long>({want, (long long)kMaxSplits + 1, (nb + 3) / 4}));
@@ -405,12 +428,12 @@ static int step_typed(const still_params_t *p, char *state, const still_state_la
             STILL_CUDA(ensure_dynamic_smem((const void *)step_attend_mma_kernel<64>, AttendPlan<64>::kTotal));
             step_attend_mma_kernel<64><<<grid, 128, AttendPlan<64>::kTotal, st>>>(
                 (const __nv_bfloat16 *)kc, (const __nv_bfloat16 *)vc, smask, (const __nv_bfloat16 *)q, part, hdr, p->H, p->Hkv,
-                cap, C, lam, t, n_splits, kMaxSplits + 1, scale_log2);
+                cap, kvr, C, lam, t, first_pos, n_splits, kMaxSplits + 1, scale_log2);
         } else {
             STILL_CUDA(ensure_dynamic_smem((const void *)step_attend_mma_kernel<128>, AttendPlan<128>::kTotal));
             step_attend_mma_kernel<128><<<grid, 128, AttendPlan<128>::kTotal, st>>>(
                 (const __nv_bfloat16 *)kc, (const __nv_bfloat16 *)vc, smask, (const __nv_bfloat16 *)q, part, hdr, p->H, p->Hkv,
-                cap, C, lam, t, n_splits, kMaxSplits + 1, scale_log2);
+                cap, kvr, C, lam, t, first_pos, n_splits, kMaxSplits + 1, scale_log2);
         }
         profile_mark_end(st);
         ++*launches;

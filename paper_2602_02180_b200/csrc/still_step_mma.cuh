@@ -64,14 +64,14 @@ struct AttendPlan {
     static constexpr int kTotal = 4 * kWarp;
 };
 
-// grid (n_splits, Hkv, B), 128 threads.  part: [B*H][max_splits][D + 2] = running max (natural
+// grid (n_splits, Hkv, B), 128 threads.  first_pos: a multiple of the chunk size.  part: [B*H][max_splits][D + 2] = running max (natural
 // log units), sum, numerator.
 template <int D>
 __global__ void __launch_bounds__(128)
 step_attend_mma_kernel(const __nv_bfloat16 *__restrict__ kc, const __nv_bfloat16 *__restrict__ vc,
                        const uint32_t *__restrict__ sel_mask, const __nv_bfloat16 *__restrict__ q,
-                       float *__restrict__ part, const int32_t *__restrict__ hdr, int H, int Hkv, long long cap, int C,
-                       int lam, long long t, int n_splits, int max_splits, float scale_log2) {
+                       float *__restrict__ part, const int32_t *__restrict__ hdr, int H, int Hkv, long long cap, long long kvr, int C,
+                       int lam, long long t, long long first_pos, int n_splits, int max_splits, float scale_log2) {
     using P = AttendPlan<D>;
     extern __shared__ __align__(16) uint8_t attend_smem[];
     if (hdr[14] != 0) return;   // the step's first kernel found the state not to match the call
@@ -79,16 +79,20 @@ step_attend_mma_kernel(const __nv_bfloat16 *__restrict__ kc, const __nv_bfloat16
     const int split = blockIdx.x, kv = blockIdx.y, b = blockIdx.z, rep = H / Hkv;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, tig = lane & 3;          // fragment row (and row + 8), column pair
-    const __nv_bfloat16 *kh = kc + ((long long)b * Hkv + kv) * cap * D;
-    const __nv_bfloat16 *vh = vc + ((long long)b * Hkv + kv) * cap * D;
+    // K / V rows live in a ring of kvr rows per KV head (position p in row p % kvr; kvr is a multiple of the chunk
+    // size, so a 32-position block never straddles the end)
+    const __nv_bfloat16 *kh = kc + ((long long)b * Hkv + kv) * kvr * D;
+    const __nv_bfloat16 *vh = vc + ((long long)b * Hkv + kv) * kvr * D;
     uint8_t *my = smem + warp * P::kWarp;
 
     const long long c_cur = t / C;
     const long long loc0 = c_cur >= 1 ? (c_cur - 1) * C : 0;   // first position of the local region
     const int n_chunk_cap = (int)(cap / C);
-    const int nb = (int)((t + 32) / 32);                         // key blocks covering positions 0..t
-    const int per = (nb + n_splits - 1) / n_splits;
-    const int kb_lo = split * per, kb_hi = min(nb, kb_lo + per);
+    // key blocks covering positions first_pos..t (first_pos > 0 with a salient-cache budget: older chunks have
+    // left the cache for the linear state)
+    const int kb0 = (int)(first_pos / 32), nb = (int)((t + 32) / 32);
+    const int per = (nb - kb0 + n_splits - 1) / n_splits;
+    const int kb_lo = kb0 + split * per, kb_hi = min(nb, kb_lo + per);
 
     // Q fragments of the group's heads (rows >= rep are zero)
     uint32_t qa[D / 16][4];
@@ -111,12 +115,13 @@ step_attend_mma_kernel(const __nv_bfloat16 *__restrict__ kc, const __nv_bfloat16
     auto load_block = [&](int kb, int stage) {
         uint8_t *ks = my + stage * P::kStage, *vs = ks + P::kTile;
         constexpr int kChunksPerRow = D / 8;
+        const long long p0 = (long long)kb * 32;
+        const long long r0 = p0 % kvr;   // ring row of the block's first position (one division per block)
 #pragma unroll
         for (int i = lane; i < 32 * kChunksPerRow; i += 32) {
             const int row = i / kChunksPerRow, ch = i % kChunksPerRow;
-            const long long pos = (long long)kb * 32 + row;
-            const bool valid = pos <= t;   // rows after the new token are zero-filled, never read from memory
-            const long long src = (valid ? pos : 0) * D + ch * 8;
+            const bool valid = p0 + row <= t;   // rows after the new token are zero-filled, never read from memory
+            const long long src = (valid ? r0 + row : 0) * D + ch * 8;
             cp_async16(ks + row * P::kRow + ch * 16, kh + src, valid);
             cp_async16(vs + row * P::kRow + ch * 16, vh + src, valid);
         }

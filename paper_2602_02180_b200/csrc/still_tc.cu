@@ -78,7 +78,8 @@ static_assert(SmemPlan<128>::kK == SmemPlan<128>::kQ + 2 * SmemPlan<128>::kTileB
 
 // Per-CTA description of the key stream.
 struct Stream {
-    int n_sel_a, n_sel_b;   // SEL tiles used by tile A / tile B
+    int sel_first;          // first SEL tile of the stream (0 unless the salient cache has a budget)
+    int n_sel_a, n_sel_b;   // SEL tiles used by tile A / tile B, counted from sel_first
     int m0;                 // first LOC tile index of interest is m0 - 1
     int has_prev;           // m0 > 0
     int has_b;              // tile B has rows below N
@@ -93,10 +94,13 @@ struct Stream {
     }
 };
 
-__device__ __forceinline__ int sel_limit(long long pos, int C, int lam) {  // visible prefix of K_sel
+__device__ __forceinline__ int sel_limit(long long pos, int C, int lam) {  // end of the visible range of K_sel
     long long c = pos / C;
     return c >= 2 ? (int)((c - 1) * lam) : 0;
 }
+// Start of the visible range: 0, or with a salient-cache budget of `budget` tokens per head (a multiple of lam;
+// the oldest cached tokens have left for the linear state) the last `budget` entries before the end.
+__device__ __forceinline__ int sel_start(int limit, int budget) { return budget > 0 ? max(limit - budget, 0) : 0; }
 
 // ---------------------------------------------------------------------------
 // Softmax warps of the attention kernels (one warpgroup per query tile, a thread per query row) and the
@@ -112,7 +116,8 @@ __device__ __forceinline__ void softmax_role(const StreamT &st, const int x, con
                                              int *status, uint8_t *stage_tile, const __nv_bfloat16 *__restrict__ y_part,
                                              const float *__restrict__ d_part, const int n_parts, const long long part_stride_y,
                                              const long long part_stride_d, __nv_bfloat16 *__restrict__ Y, const int bh,
-                                             const int N, const int C, const int lam, const float scale_log2) {
+                                             const int N, const int C, const int lam, const int budget,
+                                             const float scale_log2) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     auto col_s = [](int xx) -> uint32_t { return (uint32_t)xx * 128u; };
     auto col_o = [](int xx) -> uint32_t { return 256u + (uint32_t)xx * (uint32_t)D; };
@@ -127,7 +132,7 @@ __device__ __forceinline__ void softmax_role(const StreamT &st, const int x, con
         const uint32_t lane_addr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
         const int tq = min(t, N - 1);              // rows past N mimic the last row (never stored)
         const int c = tq / C;
-        const int lim_sel = c >= 2 ? (c - 1) * lam : 0;
+        const int lim_sel = c >= 2 ? (c - 1) * lam : 0, lo_sel = sel_start(lim_sel, budget);
         const int loc_lo = c >= 1 ? (c - 1) * C : 0;
         float m_used = -INFINITY, l_sum = 0.f;     // log2 domain
         int n_seen = 0, prev_i = -1;
@@ -137,8 +142,8 @@ __device__ __forceinline__ void softmax_role(const StreamT &st, const int x, con
             // visible column interval [lo, hi] of this row in stream tile i
             int lo, hi;
             if (st.is_sel(i)) {
-                lo = 0;
-                hi = lim_sel - i * kBlockN - 1;
+                lo = lo_sel - (st.sel_first + i) * kBlockN;
+                hi = lim_sel - (st.sel_first + i) * kBlockN - 1;
             } else {
                 const int p0 = st.loc_m(i) * kBlockN;
                 lo = loc_lo - p0;
@@ -332,7 +337,7 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                    const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_ksel,
                    const __grid_constant__ CUtensorMap tm_vsel, const __nv_bfloat16 *__restrict__ y_part,
                    const float *__restrict__ d_part, int n_parts, __nv_bfloat16 *__restrict__ Y, int *status, int H, int Hkv,
-                   int N, int C, int lam, int sel_rows, int sel_identity, float scale_log2, int n_qblocks) {
+                   int N, int C, int lam, int budget, int sel_rows, int sel_identity, float scale_log2, int n_qblocks) {
     using P = SmemPlan<D>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -358,8 +363,9 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     st.has_b = (R0 + kBlockM) < N;
     {
         int last_a = min(R0 + kBlockM - 1, N - 1), last_b = min(R0 + 2 * kBlockM - 1, N - 1);
-        st.n_sel_a = (sel_limit(last_a, C, lam) + kBlockN - 1) / kBlockN;
-        st.n_sel_b = st.has_b ? (sel_limit(last_b, C, lam) + kBlockN - 1) / kBlockN : st.n_sel_a;
+        st.sel_first = sel_start(sel_limit(R0, C, lam), budget) / kBlockN;   // the CTA's first row sees the oldest entries
+        st.n_sel_a = max((sel_limit(last_a, C, lam) + kBlockN - 1) / kBlockN - st.sel_first, 0);
+        st.n_sel_b = st.has_b ? max((sel_limit(last_b, C, lam) + kBlockN - 1) / kBlockN - st.sel_first, 0) : st.n_sel_a;
     }
     st.n_tiles = st.n_sel_b + st.has_prev + 1 + st.has_b;
 
@@ -416,7 +422,7 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     const int i = armed_k, ks = i % P::kKStages;
                     if (mbar_try_wait(k_empty + ks, ((i / P::kKStages) & 1) ^ 1)) {
                         const bool sel = st.is_sel(i);
-                        const int row = sel ? sel_base + i * kBlockN : (b * Hkv + kvh) * N + st.loc_m(i) * kBlockN;
+                        const int row = sel ? sel_base + (st.sel_first + i) * kBlockN : (b * Hkv + kvh) * N + st.loc_m(i) * kBlockN;
                         mbar_expect_tx(k_full + ks, P::kTileBytes);
                         for (int half = 0; half < D / 64; ++half)
                             tma_load_2d(smem + P::kK + ks * P::kTileBytes + half * (kBlockN * 128), sel ? &tm_ksel : &tm_k,
@@ -429,7 +435,7 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     const int i = armed_v, vs = i % P::kVStages;
                     if (mbar_try_wait(v_empty + vs, ((i / P::kVStages) & 1) ^ 1)) {
                         const bool sel = st.is_sel(i);
-                        const int row = sel ? sel_base + i * kBlockN : (b * Hkv + kvh) * N + st.loc_m(i) * kBlockN;
+                        const int row = sel ? sel_base + (st.sel_first + i) * kBlockN : (b * Hkv + kvh) * N + st.loc_m(i) * kBlockN;
                         mbar_expect_tx(v_full + vs, P::kTileBytes);
                         for (int half = 0; half < D / 64; ++half)
                             tma_load_2d(smem + P::kV + vs * P::kTileBytes + half * (kBlockN * 128), sel ? &tm_vsel : &tm_v,
@@ -547,7 +553,7 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         softmax_role<D, P::kKStages, P::kVStages, false>(st, x, R0 + x * kBlockM, tmem_base, s_full, k_empty, v_empty, p_half, 0u,
                                                          o_final, abort_flag, status, smem + P::kQ + x * P::kTileBytes, y_part,
                                                          d_part, n_parts, (long long)gridDim.y * N * D, (long long)gridDim.y * N,
-                                                         Y, bh, N, C, lam, scale_log2);
+                                                         Y, bh, N, C, lam, budget, scale_log2);
     }
     tc_fence_before();
     __syncthreads();
@@ -593,7 +599,7 @@ static_assert(PairPlan<128>::kAlloc <= kMaxDynamicSmem, "pair attention kernel: 
 
 // Key stream of a CTA pair (same in both CTAs): SEL tiles, then the LOC tiles m_first .. m_last.
 struct PairStream {
-    int n_sel_a, n_sel_b, m0, m_first, has_b, n_tiles;
+    int sel_first, n_sel_a, n_sel_b, m0, m_first, has_b, n_tiles;   // SEL tiles are counted from sel_first
     __device__ __forceinline__ bool is_sel(int i) const { return i < n_sel_b; }
     __device__ __forceinline__ int loc_m(int i) const { return m_first + (i - n_sel_b); }
     __device__ __forceinline__ bool used_by(int x, int i) const {
@@ -609,7 +615,7 @@ sa_merge_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                      const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_ksel,
                      const __grid_constant__ CUtensorMap tm_vsel, const __nv_bfloat16 *__restrict__ y_part,
                      const float *__restrict__ d_part, int n_parts, __nv_bfloat16 *__restrict__ Y, int *status, int H, int Hkv, int N,
-                     int C, int lam, int sel_rows, int sel_identity, float scale_log2, int n_pairs) {
+                     int C, int lam, int budget, int sel_rows, int sel_identity, float scale_log2, int n_pairs) {
     using P = PairPlan<D>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -637,8 +643,9 @@ sa_merge_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     st.has_b = (R0 + 2 * kBlockM) < N;
     {
         const int last_a = min(R0 + 2 * kBlockM - 1, N - 1), last_b = min(R0 + 4 * kBlockM - 1, N - 1);
-        st.n_sel_a = (sel_limit(last_a, C, lam) + kBlockN - 1) / kBlockN;
-        st.n_sel_b = st.has_b ? (sel_limit(last_b, C, lam) + kBlockN - 1) / kBlockN : st.n_sel_a;
+        st.sel_first = sel_start(sel_limit(R0, C, lam), budget) / kBlockN;   // the pair's first row sees the oldest entries
+        st.n_sel_a = max((sel_limit(last_a, C, lam) + kBlockN - 1) / kBlockN - st.sel_first, 0);
+        st.n_sel_b = st.has_b ? max((sel_limit(last_b, C, lam) + kBlockN - 1) / kBlockN - st.sel_first, 0) : st.n_sel_a;
         const int m_last = min(st.m0 + (st.has_b ? 3 : 1), (N - 1) / kBlockN);
         st.n_tiles = st.n_sel_b + (m_last - st.m_first + 1);
     }
@@ -701,7 +708,7 @@ sa_merge_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     const int i = armed_k, ks = i % P::kKStages;
                     if (mbar_try_wait(k_empty + ks, ((i / P::kKStages) & 1) ^ 1)) {
                         const bool sel = st.is_sel(i);
-                        const int row = (sel ? sel_base + i * kBlockN : (b * Hkv + kvh) * N + st.loc_m(i) * kBlockN) +
+                        const int row = (sel ? sel_base + (st.sel_first + i) * kBlockN : (b * Hkv + kvh) * N + st.loc_m(i) * kBlockN) +
                                         (int)rank * (kBlockN / 2);   // this CTA's 64 keys
                         if (rank == 0) mbar_expect_tx(k_full + ks, 2 * P::kKHalf);
                         for (int half = 0; half < D / 64; ++half)
@@ -715,7 +722,7 @@ sa_merge_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     const int i = armed_v, vs = i % P::kVStages;
                     if (mbar_try_wait(v_empty + vs, ((i / P::kVStages) & 1) ^ 1)) {
                         const bool sel = st.is_sel(i);
-                        const int row = sel ? sel_base + i * kBlockN : (b * Hkv + kvh) * N + st.loc_m(i) * kBlockN;
+                        const int row = sel ? sel_base + (st.sel_first + i) * kBlockN : (b * Hkv + kvh) * N + st.loc_m(i) * kBlockN;
                         if (rank == 0) mbar_expect_tx(v_full + vs, 2 * P::kVHalf);
                         for (int q = 0; q < D / 128; ++q)           // this CTA's D / 2 value columns, 64 at a time
                             tma_load_2d_pair(smem + P::kV + vs * P::kVHalf + q * (kBlockN * 128), sel ? &tm_vsel : &tm_v,
@@ -842,7 +849,7 @@ sa_merge_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                                                         k_empty, v_empty, p_half, mapa(smem_u32(p_half), 0), o_final,
                                                         abort_flag, status, smem + P::kQ + x * P::kQTile, y_part, d_part, n_parts,
                                                         (long long)gridDim.y * N * D, (long long)gridDim.y * N, Y, bh, N, C, lam,
-                                                        scale_log2);
+                                                        budget, scale_log2);
         if (*abort_flag) tell_peer();
     }
     // Nobody touches the peer's shared memory or tensor memory after this point.
@@ -1225,7 +1232,7 @@ int launch_tc(const still_params_t *p, long long N, const void *Q, const void *K
         dim3 grid((unsigned)(2 * n_pairs), (unsigned)BH);   // clusters of two along x
         profile_mark_begin(st);
         sa_merge_pair_kernel<D><<<grid, kThreads, PairPlan<D>::kAlloc, st>>>(
-            tq, tk, tv, tks, tvs, (const bf *)y_part, d_part, n_parts, (bf *)Y, status, p->H, p->Hkv, (int)N, p->chunk, p->topk, (int)sel_rows,
+            tq, tk, tv, tks, tvs, (const bf *)y_part, d_part, n_parts, (bf *)Y, status, p->H, p->Hkv, (int)N, p->chunk, p->topk, (int)p->max_salient, (int)sel_rows,
             identity ? 1 : 0, scale_log2, n_pairs);
         profile_mark_end(st);
     } else {
@@ -1234,7 +1241,7 @@ int launch_tc(const still_params_t *p, long long N, const void *Q, const void *K
         dim3 grid((unsigned)n_qblocks, (unsigned)BH);
         profile_mark_begin(st);
         sa_merge_tc_kernel<D><<<grid, kThreads, SmemPlan<D>::kAlloc, st>>>(
-            tq, tk, tv, tks, tvs, (const bf *)y_part, d_part, n_parts, (bf *)Y, status, p->H, p->Hkv, (int)N, p->chunk, p->topk, (int)sel_rows,
+            tq, tk, tv, tks, tvs, (const bf *)y_part, d_part, n_parts, (bf *)Y, status, p->H, p->Hkv, (int)N, p->chunk, p->topk, (int)p->max_salient, (int)sel_rows,
             identity ? 1 : 0, scale_log2, n_qblocks);
         profile_mark_end(st);
     }

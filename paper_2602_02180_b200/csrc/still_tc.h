@@ -72,6 +72,9 @@ int tc_la_segments(const still_params_t *p, long long N, int *seg_chunks);
 
 // ---- decode step ----------------------------------------------------------------------
 size_t step_scratch_bytes(const still_params_t *p, long long capacity);
+// Rows of the K / V store per KV head in a decode state of that capacity: the capacity itself, or, with a
+// salient-cache budget, a ring that holds the cached chunks, the two-chunk local region and the chunk being routed.
+long long state_kv_rows(const still_params_t *p, long long capacity);
 int step_launch(const still_params_t *p, char *state, const still_state_layout_t *L, long long t_pos,
                 const void *q, const void *k, const void *v, const void *g, const void *Wq,
                 const void *bq, const void *Wk, const void *bk, void *y, cudaStream_t st,

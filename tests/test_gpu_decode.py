@@ -12,7 +12,7 @@ from tests import util_parity as U
 pytestmark = pytest.mark.gpu
 
 
-def _decode_case(w, n0, n_steps, gate=False, tweak=None, expect_ties=False, n_heads=4, want_y=True):
+def _decode_case(w, n0, n_steps, gate=False, tweak=None, expect_ties=False, n_heads=4, want_y=True, max_salient=0):
     """Prefill n0 tokens into a state, decode n_steps more, compare every decoded row of the sampled heads
     with the oracle's chunk-wise form over the whole sequence (the GPU's selection forced)."""
     dev = "cuda"
@@ -32,7 +32,7 @@ def _decode_case(w, n0, n_steps, gate=False, tweak=None, expect_ties=False, n_he
     step_in = [t[:, :, n0:].permute(2, 0, 1, 3).contiguous() if t is not None else None for t in (Q, K, V, G)]  # [steps,B,heads,d]
     pre = [t[:, :, :n0].contiguous() if t is not None else None for t in (Q, K, V, G)]
     del Q, K, V, G
-    p = U.params_of(w)
+    p = U.params_of(w, max_salient=max_salient)
     cap = N + 5
     lay = still.state_layout(p, cap)
     state = torch.zeros(lay["total"], dtype=torch.uint8, device=dev)
@@ -66,7 +66,7 @@ def _decode_case(w, n0, n_steps, gate=False, tweak=None, expect_ties=False, n_he
     if lam > 0:
         sel = state[lay["sel_idx"]: lay["sel_idx"] + w.B * w.H * capT * lam * 4].view(torch.int32).view(w.B, w.H, capT, lam)
     rows = list(range(n0, N))
-    hp = oracle.HeadParams(C, lam, w.sm_scale)
+    hp = oracle.HeadParams(C, lam, w.sm_scale, max_salient=max_salient)
     tie_seen = False
     worst = 0.0
     for b, h in heads:
@@ -111,6 +111,30 @@ def _decode_case(w, n0, n_steps, gate=False, tweak=None, expect_ties=False, n_he
 def test_decode_matches_oracle(dtype, B, H, Hkv, d, C, k, n0, steps):
     w = synth.Workload("t", B, H, Hkv, d, n0, C, k, dtype, "iid", 999)
     _decode_case(w, n0, steps, gate=(k not in (0, C)))
+
+
+@pytest.mark.parametrize("B,H,Hkv,d,C,k,budget,n0,steps", [
+    (1, 4, 2, 128, 64, 16, 48, 64 * 7 + 11, 64 * 3 + 9),     # prefill already past the budget, three routings while decoding
+    (2, 2, 1, 64, 64, 8, 16, 72, 64 * 7),                    # the budget is reached during the decode
+    (1, 2, 2, 128, 64, 64, 128, 64 * 5, 64 * 2 + 5),         # every token selected: sliding window + linear state
+    (1, 2, 1, 64, 64, 8, 8, 0, 64 * 6),                      # from an empty state
+])
+def test_decode_with_a_salient_cache_budget(B, H, Hkv, d, C, k, budget, n0, steps):
+    # Tokens that a newly routed chunk pushes out of the capped salient cache are folded into (S, z) at that step,
+    # and the split-KV pass reads only the chunks still cached.
+    w = synth.Workload("t", B, H, Hkv, d, n0, C, k, "bf16", "iid", 4711)
+    _decode_case(w, n0, steps, gate=True, max_salient=budget)
+
+
+def test_budgeted_state_size_does_not_grow_with_the_sequence():
+    # with a budget the K / V store of the state is a ring over the cached chunks, the local region and the chunk
+    # being routed; what still grows with the capacity are 4-byte scores and the per-chunk index tables
+    free = still.StillParams(8, 32, 8, 128, 64, 16)
+    capped = still.StillParams(8, 32, 8, 128, 64, 16, max_salient=448)
+    small, big = still.state_bytes(capped, 4096), still.state_bytes(capped, 65536)
+    assert still.state_bytes(free, 65536) > 12 * still.state_bytes(free, 4096) > 0
+    kv_ring = 8 * 8 * (448 // 16 + 3) * 64 * 128 * 2 * 2
+    assert big - small < 0.1 * still.state_bytes(free, 65536) and small > kv_ring and big < 3 * small
 
 
 @pytest.mark.parametrize("k", [64, 16])

@@ -52,6 +52,39 @@ def test_small_shapes(dtype, B, H, Hkv, d, N, C, k):
                     G=r["G"], bq=r["bq"], bk=r["bk"])
 
 
+@pytest.mark.parametrize(
+    "B,H,Hkv,d,N,C,k,budget",
+    [
+        (1, 4, 2, 128, 64 * 12 + 9, 64, 16, 48),      # three chunks' selections stay cached
+        (2, 2, 1, 64, 128 * 9 + 40, 128, 32, 64),     # two sub-chunks per chunk
+        (1, 2, 2, 128, 64 * 10 + 3, 64, 64, 128),     # every token selected: a sliding window of two chunks + linear state
+        (1, 2, 1, 128, 64 * 40 + 17, 64, 16, 64),     # the state scan in four segments
+        (1, 4, 2, 128, 64 * 9, 64, 16, 16 * 64),      # a budget that is never reached
+        (1, 2, 2, 64, 64 * 30, 64, 8, 8),             # a single chunk's selections
+    ],
+)
+def test_salient_cache_budget(B, H, Hkv, d, N, C, k, budget):
+    # max_salient: per head at most `budget` selected tokens stay in the softmax branch; the oldest leave for the
+    # linear state when a newly routed chunk pushes them out (this library's rule; the paper caps the cache
+    # without stating one).  The oracle applies the same rule.
+    w = _small("t", "bf16", B, H, Hkv, d, N, C, k)
+    r = U.run_prefill(w, gate=True, max_salient=budget)
+    heads = U.sample_heads(w, 4)
+    U.check_selection(r["scores"], r["sel"], C, k, heads)
+    U.check_outputs(w, r["Q"], r["K"], r["V"], r["Wq"], r["Wk"], r["Y"], r["scores"], r["sel"], heads, G=r["G"],
+                    max_salient=budget)
+    if budget >= (N // C) * k:   # never reached: the same bits as without a budget
+        free = U.run_prefill(w, gate=True)
+        assert torch.equal(free["Y"], r["Y"])
+
+
+def test_salient_cache_budget_must_be_whole_chunks_of_selections():
+    p = still.StillParams(1, 2, 2, 64, 64, 16, max_salient=40)
+    assert still.workspace_bytes(p, 256) == 0
+    assert still.workspace_bytes(still.StillParams(1, 2, 2, 64, 64, 16, torch.float32, max_salient=32), 256) == 0   # FMA path
+    assert still.workspace_bytes(still.StillParams(1, 2, 2, 64, 64, 16, max_salient=32), 256) > 0
+
+
 def _has_tie(scores, C):
     """True when some chunk holds two equal finite scores (so the tie arm of the ranking decided)."""
     sc = scores.cpu().numpy()

@@ -43,7 +43,7 @@ def jaccard(a, b):
 
 
 def check_outputs(w, Q, K, V, Wq, Wk, Y, scores, sel_idx, heads, rows=None, G=None, bq=None, bk=None,
-                  tol=None, eps=1e-6, score_tol=None, report=None):
+                  tol=None, eps=1e-6, score_tol=None, report=None, max_salient=0):
     """Y of the sampled heads (and rows) against the oracle run with the GPU's selection, and the GPU's
     scores against the oracle's.  Returns (worst Y error, worst score error); `report`, if a dict, also
     receives the Jaccard agreement between the oracle's own selection and the GPU's (reported, not gated:
@@ -51,7 +51,7 @@ def check_outputs(w, Q, K, V, Wq, Wk, Y, scores, sel_idx, heads, rows=None, G=No
     tol = TOL[w.torch_dtype] if tol is None else tol
     score_tol = SCORE_TOL[w.torch_dtype] if score_tol is None else score_tol
     rep = w.H // w.Hkv
-    p = oracle.HeadParams(w.C, w.k, w.sm_scale, eps)
+    p = oracle.HeadParams(w.C, w.k, w.sm_scale, eps, max_salient=max_salient)
     worst = 0.0
     score_err = 0.0
     for b, h in heads:
@@ -76,7 +76,7 @@ def check_outputs(w, Q, K, V, Wq, Wk, Y, scores, sel_idx, heads, rows=None, G=No
     return worst, score_err
 
 
-def run_prefill(w, device="cuda", gate=False, bias=False, **fwd_kw):
+def run_prefill(w, device="cuda", gate=False, bias=False, max_salient=0, **fwd_kw):
     Q, K, V = synth.make_qkv(w, device)
     Wq, Wk = synth.make_npmap_weights(w, device)
     G = synth.make_gate(w, device) if gate else None
@@ -85,7 +85,7 @@ def run_prefill(w, device="cuda", gate=False, bias=False, **fwd_kw):
         g = torch.Generator(device=device).manual_seed(w.seed + 77)
         bq = (torch.randn(w.H, w.d_f, generator=g, device=device) * 0.05).to(w.torch_dtype)
         bk = (torch.randn(w.Hkv, w.d_f, generator=g, device=device) * 0.05).to(w.torch_dtype)
-    p = params_of(w)
+    p = params_of(w, max_salient=max_salient)
     Y, scores, sel = still.hybrid_attn_fwd(p, Q, K, V, Wq, Wk, G=G, bq=bq, bk=bk, **fwd_kw)
     torch.cuda.synchronize()
     return dict(p=p, Q=Q, K=K, V=V, Wq=Wq, Wk=Wk, G=G, bq=bq, bk=bk, Y=Y, scores=scores, sel=sel)
