@@ -5,10 +5,10 @@
 // m16n8k16 tensor-core tile, so the K / V rows are read once for the whole group.  Which rows a
 // query head sees is a per-head membership mask: for a position in a routed chunk, whether the
 // head's selection (the sel_mask words of the decode state) contains it; for the two-chunk local region, every position up to the
-// new token.  Whole key blocks are streamed (coalesced 16-byte cp.async into padded shared-memory
-// rows, two stages per warp) and rows a head did not select get weight zero; with topk = chunk
-// that is exactly the salient cache, with a smaller topk a block is still read once for the
-// group rather than once per head.
+// new token.  Key blocks are streamed by 16-byte cp.async into padded shared-memory rows, two stages per
+// warp; a row is read from memory only if some head of the group selected it (the union of the group's
+// salient caches, read once for the group rather than once per head) and gets weight zero for the heads
+// that did not; with topk = chunk that is every row.
 // Each warp runs its own online softmax over its blocks; the four warps are merged through shared
 // memory and the CTA writes one partial (max, sum, numerator) per head and split.
 #pragma once
@@ -112,7 +112,9 @@ step_attend_mma_kernel(const __nv_bfloat16 *__restrict__ kc, const __nv_bfloat16
     for (int i = 0; i < D / 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
     float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};   // rows g and g + 8, log2 domain
 
-    auto load_block = [&](int kb, int stage) {
+    // Rows of a block that no query head of the group sees are not read from memory (a zero-filling copy with
+    // no source bytes): with topk < chunk only the union of the group's selections crosses HBM.
+    auto load_block = [&](int kb, int stage, uint32_t rows_needed) {
         uint8_t *ks = my + stage * P::kStage, *vs = ks + P::kTile;
         constexpr int kChunksPerRow = D / 8;
         const long long p0 = (long long)kb * 32;
@@ -120,45 +122,46 @@ step_attend_mma_kernel(const __nv_bfloat16 *__restrict__ kc, const __nv_bfloat16
 #pragma unroll
         for (int i = lane; i < 32 * kChunksPerRow; i += 32) {
             const int row = i / kChunksPerRow, ch = i % kChunksPerRow;
-            const bool valid = p0 + row <= t;   // rows after the new token are zero-filled, never read from memory
+            const bool valid = (rows_needed >> row) & 1u;
             const long long src = (valid ? r0 + row : 0) * D + ch * 8;
             cp_async16(ks + row * P::kRow + ch * 16, kh + src, valid);
             cp_async16(vs + row * P::kRow + ch * 16, vh + src, valid);
         }
     };
+    // Membership word of block kb for the head in this lane (lanes >= group size: 0): bit j = position 32 kb + j is
+    // visible to the head.  Local region: every position up to the new token; routed chunks: the head's selection
+    // (bit masks written when the chunk was routed), all of it when topk = chunk.
+    auto member_word = [&](int kb) -> uint32_t {
+        if (kb >= kb_hi || lane >= rep) return 0u;
+        const long long p0 = (long long)kb * 32;
+        if (p0 >= loc0) {
+            const long long last = t - p0;   // positions up to the new token
+            return last >= 31 ? 0xffffffffu : ((1u << (int)(last + 1)) - 1u);
+        }
+        if (lam >= C) return 0xffffffffu;
+        if (lam <= 0) return 0u;
+        const int chunk = (int)(p0 / C), word = (int)((p0 % C) / 32);
+        return sel_mask[(((long long)b * H + (long long)kv * rep + lane) * n_chunk_cap + chunk) * (C / 32) + word];
+    };
 
+    // The membership words run two blocks ahead of the compute and one ahead of the copies they steer.
     const int first = kb_lo + warp;
-    if (first < kb_hi) load_block(first, 0);
+    uint32_t m_cur = member_word(first), m_next = member_word(first + 4);
+    if (first < kb_hi) load_block(first, 0, __reduce_or_sync(0xffffffffu, m_cur));
     cp_async_commit();
     int it = 0;
     for (int kb = first; kb < kb_hi; kb += 4, ++it) {
         const int stage = it & 1;
-        if (kb + 4 < kb_hi) load_block(kb + 4, stage ^ 1);
+        const uint32_t m_after = member_word(kb + 8);
+        if (kb + 4 < kb_hi) load_block(kb + 4, stage ^ 1, __reduce_or_sync(0xffffffffu, m_next));
         cp_async_commit();
 
         // membership of the block's 32 positions for rows g and g + 8 (bit j: position 32 kb + j)
-        uint32_t vis[2] = {0u, 0u};
-        {
-            const long long p0 = (long long)kb * 32;
-            if (p0 >= loc0) {
-                const long long last = t - p0;   // positions up to the new token
-                const uint32_t mloc = last >= 31 ? 0xffffffffu : ((1u << (int)(last + 1)) - 1u);
-                vis[0] = g < rep ? mloc : 0u;
-                vis[1] = g + 8 < rep ? mloc : 0u;
-            } else if (lam >= C) {
-                vis[0] = g < rep ? 0xffffffffu : 0u;   // every token of a routed chunk was selected
-                vis[1] = g + 8 < rep ? 0xffffffffu : 0u;
-            } else if (lam > 0) {
-                // selection of the block's chunk as bit masks (written when the chunk was routed): lane r
-                // fetches the word of head r, rows g and g + 8 take theirs by shuffle
-                const int chunk = (int)(p0 / C), word = (int)((p0 % C) / 32);
-                uint32_t mine = 0u;
-                if (lane < rep)
-                    mine = sel_mask[(((long long)b * H + (long long)kv * rep + lane) * n_chunk_cap + chunk) * (C / 32) + word];
-                vis[0] = __shfl_sync(0xffffffffu, mine, g);
-                vis[1] = __shfl_sync(0xffffffffu, mine, g + 8);
-            }
-        }
+        uint32_t vis[2];
+        vis[0] = __shfl_sync(0xffffffffu, m_cur, g);
+        vis[1] = __shfl_sync(0xffffffffu, m_cur, g + 8);
+        m_cur = m_next;
+        m_next = m_after;
         cp_async_wait<1>();
         __syncwarp();
         const uint8_t *ks = my + stage * P::kStage, *vs = ks + P::kTile;
