@@ -132,16 +132,16 @@ __device__ __forceinline__ void npmap_row(const float *xw, const TW *W, const TW
     nx2 = warp_sum(nx2);
     float f[4], nf2 = 0.f;
 #pragma unroll
-    for (int jj = 0; jj < 4; ++jj) {
-        f[jj] = 0.f;
-        if (jj < jpl) {
-            int j = lane + 32 * jj;
-            float acc = bias ? ld_f(bias + j) : 0.f;
-            for (int i = 0; i < d; ++i) acc = fmaf(xw[i], ld_f(W + i * df + j), acc);
-            f[jj] = acc;
-            nf2 += acc * acc;
-        }
+    for (int jj = 0; jj < 4; ++jj) f[jj] = (jj < jpl && bias) ? ld_f(bias + lane + 32 * jj) : 0.f;
+    for (int i = 0; i < d; ++i) {   // one read of x_i serves the lane's (up to) four outputs
+        const float xi = xw[i];
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj)
+            if (jj < jpl) f[jj] = fmaf(xi, ld_f(W + i * df + lane + 32 * jj), f[jj]);
     }
+#pragma unroll
+    for (int jj = 0; jj < 4; ++jj)
+        if (jj < jpl) nf2 += f[jj] * f[jj];
     nf2 = warp_sum(nf2);
     const float ratio = sqrtf(nx2) / fmaxf(sqrtf(nf2), 1e-12f);
     float umax = -INFINITY, umin = INFINITY;

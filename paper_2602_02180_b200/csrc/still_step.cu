@@ -138,7 +138,8 @@ __global__ void __launch_bounds__(256)
 step_route_kernel(const T *__restrict__ kc, const T *__restrict__ vc, const float *__restrict__ score,
                   int32_t *__restrict__ sel_idx, uint32_t *__restrict__ sel_mask, float *__restrict__ S,
                   float *__restrict__ z, const T *__restrict__ Wk, const T *__restrict__ bk, const int32_t *__restrict__ hdr,
-                  int H, int Hkv, long long cap, long long kvr, int d, int df, int C, int lam, long long cr, int window) {
+                  int H, int Hkv, long long cap, long long kvr, int d, int df, int C, int lam, long long cr, int window,
+                  int w_in_smem) {
     extern __shared__ float smem[];
     if (hdr[14] != 0) return;   // the step's first kernel found the state not to match the call
     const int dp = 2 * df;
@@ -147,6 +148,7 @@ step_route_kernel(const T *__restrict__ kc, const T *__restrict__ vc, const floa
     float *xs = vs + C * d;           // [8][d]
     float *sc = xs + 8 * d;           // [C]
     int *flag = reinterpret_cast<int *>(sc + C);  // [C]
+    T *Ws = reinterpret_cast<T *>(flag + C);      // [d][df] the head's W_k (read once per row of the chunk otherwise)
     const int h = blockIdx.x, b = blockIdx.y, kv = h / (H / Hkv);
     const long long bh = (long long)b * H + h;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -165,6 +167,11 @@ step_route_kernel(const T *__restrict__ kc, const T *__restrict__ vc, const floa
     const T *Wh = Wk + (long long)kv * d * df;
     const T *bh_ = bk ? bk + (long long)kv * df : nullptr;
     float *Sh = S + bh * dp * d;
+    const T *Wuse = Wh;   // W_k from shared memory when it fits beside the chunk's tiles, else from global memory
+    if (w_in_smem && (lam < C || window > 0)) {
+        for (int i = threadIdx.x; i < d * df; i += blockDim.x) Ws[i] = Wh[i];
+        Wuse = Ws;
+    }
     // pass 0: the unselected tokens of chunk cr; pass 1: the selected tokens of the chunk that leaves the cache
     for (int pass = 0; pass < 2; ++pass) {
         const long long chunk = pass == 0 ? cr : cr - window;
@@ -185,7 +192,7 @@ step_route_kernel(const T *__restrict__ kc, const T *__restrict__ vc, const floa
             if (!flag[r]) {
                 for (int i = lane; i < d; i += 32) xw[i] = ld_f(kh + (long long)r * d + i);
                 __syncwarp();
-                npmap_row(xw, Wh, bh_, d, df, lane, ep, en);
+                npmap_row(xw, Wuse, bh_, d, df, lane, ep, en);
             }
 #pragma unroll
             for (int jj = 0; jj < 4; ++jj)
@@ -201,11 +208,30 @@ step_route_kernel(const T *__restrict__ kc, const T *__restrict__ vc, const floa
             __syncwarp();
         }
         __syncthreads();
-        for (int idx = threadIdx.x; idx < dp * d; idx += blockDim.x) {
-            int f = idx / d, e = idx - f * d;
-            float acc = Sh[idx];
-            for (int i = 0; i < C; ++i) acc = fmaf(ph[i * dp + f], vs[i * d + e], acc);
-            Sh[idx] = acc;
+        // S[f][e] += sum_i phi[i][f] v[i][e]: a thread owns 4 features x 8 value columns at a time, so that a token
+        // costs 3 shared-memory reads for 32 multiply-adds
+        for (int blk = threadIdx.x; blk < (dp / 4) * (d / 8); blk += blockDim.x) {
+            const int f0 = (blk / (d / 8)) * 4, e0 = (blk % (d / 8)) * 8;
+            float acc[4][8];
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+#pragma unroll
+                for (int c = 0; c < 8; ++c) acc[a][c] = Sh[(f0 + a) * d + e0 + c];
+            for (int i = 0; i < C; ++i) {
+                const float4 pf = *reinterpret_cast<const float4 *>(ph + i * dp + f0);
+                const float4 v0 = *reinterpret_cast<const float4 *>(vs + i * d + e0);
+                const float4 v1 = *reinterpret_cast<const float4 *>(vs + i * d + e0 + 4);
+                const float pa[4] = {pf.x, pf.y, pf.z, pf.w};
+                const float vv[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+#pragma unroll
+                for (int a = 0; a < 4; ++a)
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) acc[a][c] = fmaf(pa[a], vv[c], acc[a][c]);
+            }
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+#pragma unroll
+                for (int c = 0; c < 8; ++c) Sh[(f0 + a) * d + e0 + c] = acc[a][c];
         }
         for (int f = threadIdx.x; f < dp; f += blockDim.x) {
             float acc = z[bh * dp + f];
@@ -401,10 +427,12 @@ static int step_typed(const still_params_t *p, char *state, const still_state_la
     const long long c_cur = t / C;
     if (t % C == 0 && c_cur >= 2) {
         size_t smem = ((size_t)C * 2 * df + (size_t)C * d + 8 * (size_t)d + C) * 4 + (size_t)C * 4;
+        const int w_in_smem = smem + (size_t)d * df * sizeof(T) <= 200 * 1024 ? 1 : 0;
+        if (w_in_smem) smem += (size_t)d * df * sizeof(T);
         STILL_CUDA(cudaFuncSetAttribute(step_route_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)smem));
         step_route_kernel<T><<<dim3(p->H, p->B), 256, smem, st>>>(kc, vc, score, sel, smask, S, z, Wk, bk, hdr, p->H,
-                                                                  p->Hkv, cap, kvr, d, df, C, lam, c_cur - 2, window);
+                                                                  p->Hkv, cap, kvr, d, df, C, lam, c_cur - 2, window, w_in_smem);
         ++*launches;
         STILL_CUDA(cudaGetLastError());
     }
