@@ -42,6 +42,10 @@
 #include "still_common.cuh"
 #include "still_tc_ptx.cuh"
 
+#ifndef STILL_POLY_OF4
+#define STILL_POLY_OF4 1
+#endif
+
 namespace still {
 
 namespace {
@@ -109,7 +113,7 @@ __device__ __forceinline__ int sel_start(int limit, int budget) { return budget 
 // epilogue's staging space).  The barriers are this CTA's, except that in a CTA pair the two halves of P
 // are announced on the first CTA's p_half barriers (p_half_cluster: their address in the cluster window).
 // ---------------------------------------------------------------------------
-template <int D, int kKStages, int kVStages, bool kPair, class StreamT>
+template <int D, int kKStages, int kVStages, bool kPair, int kPolyOf4, class StreamT>
 __device__ __forceinline__ void softmax_role(const StreamT &st, const int x, const int tile_row0, const uint32_t tmem_base,
                                              uint64_t *s_full, uint64_t *k_empty, uint64_t *v_empty, uint64_t *p_half,
                                              const uint32_t p_half_cluster, uint64_t *o_final, volatile int *abort_flag,
@@ -207,11 +211,11 @@ __device__ __forceinline__ void softmax_role(const StreamT &st, const int x, con
             const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
             const float2 scale2 = make_float2(scale_log2, scale_log2), negm2 = make_float2(neg_m, neg_m);
             float2 acc = make_float2(0.f, 0.f);
-            // P = 2^(s * scale - m) as bf16 over S, in two halves of 64 columns; the MMA warp
-            // starts on the first half while the second is computed.  (All exponentials go to the
-            // MUFU unit: with a cubic 2^x on the FMA pipes for a quarter, half or three quarters of them the
-            // kernel was measured 3.6 % slower per quarter -- every added instruction of this warp costs about a
-            // cycle of the tile's serial chain.)
+            // P = 2^(s * scale - m) as bf16 over S, in two halves of 64 columns; the MMA warp starts on the first
+            // half while the second is computed.  The MUFU unit (one warp instruction per eight cycles) would need
+            // 1024 cycles for a warp's 128 exponentials of a tile, which is as long as the tensor pipe needs for the
+            // tile's two products; so kPolyOf4 of every four column pairs take 2^x from the FMA pipes instead (see
+            // exp2_fma2), interleaved with the others so that both units work at the same time.
 #pragma unroll
             for (int q = 0; q < 2; ++q) {
                 uint32_t pk[32];
@@ -219,7 +223,7 @@ __device__ __forceinline__ void softmax_role(const StreamT &st, const int x, con
                 for (int j = 0; j < 32; ++j) {
                     const float2 sv = make_float2(s[q * 64 + 2 * j], s[q * 64 + 2 * j + 1]);
                     const float2 xv = __ffma2_rn(sv, scale2, negm2);
-                    const float2 pr = make_float2(ex2(xv.x), ex2(xv.y));
+                    const float2 pr = (j % 4) < kPolyOf4 ? exp2_fma2(xv) : make_float2(ex2(xv.x), ex2(xv.y));
                     acc = __fadd2_rn(acc, pr);
                     pk[j] = pack_bf16(pr.x, pr.y);
                     if (q == 1 && j == 12) {
@@ -550,7 +554,7 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         reg_inc<216>();
         // ------------------------------------------------------------ softmax + epilogue
         const int x = (warp - 4) >> 2;                 // 0: tile A, 1: tile B
-        softmax_role<D, P::kKStages, P::kVStages, false>(st, x, R0 + x * kBlockM, tmem_base, s_full, k_empty, v_empty, p_half, 0u,
+        softmax_role<D, P::kKStages, P::kVStages, false, 0>(st, x, R0 + x * kBlockM, tmem_base, s_full, k_empty, v_empty, p_half, 0u,
                                                          o_final, abort_flag, status, smem + P::kQ + x * P::kTileBytes, y_part,
                                                          d_part, n_parts, (long long)gridDim.y * N * D, (long long)gridDim.y * N,
                                                          Y, bh, N, C, lam, budget, scale_log2);
@@ -631,8 +635,10 @@ sa_merge_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + P::kMisc + 4);
     volatile int *failed_before = reinterpret_cast<volatile int *>(smem + P::kMisc + 8);
 
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t rank = cluster_ctarank(), peer = rank ^ 1u;
+    // (warp index and cluster rank through a shuffle / from the block index: values the compiler knows to be
+    // the same in all lanes)
+    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
+    const uint32_t rank = blockIdx.x & 1u, peer = rank ^ 1u;
     const int pb = n_pairs - 1 - (int)(blockIdx.x >> 1);  // heavy blocks first
     const int bh = blockIdx.y, b = bh / H, h = bh % H, kvh = h / (H / Hkv);
     const int R0 = pb * 4 * kBlockM;
@@ -678,7 +684,7 @@ sa_merge_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     tc_fence_before();
     cluster_sync_all();   // both CTAs hold their tensor memory before the first instruction of the pair
     tc_fence_after();
-    const uint32_t tmem_base = *tmem_base_slot;
+    const uint32_t tmem_base = __shfl_sync(0xffffffffu, *tmem_base_slot, 0);
     auto col_s = [](int x) -> uint32_t { return (uint32_t)x * 128u; };
     auto col_o = [](int x) -> uint32_t { return 256u + (uint32_t)x * (uint32_t)D; };
     // a role that gives up tells the other CTA, whose waits would otherwise run to their own limit
@@ -760,7 +766,14 @@ sa_merge_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         }
     } else if (warp == 1 && rank == 0) {
         // ------------------------------------------------------------ MMA issuer (rank 0 only)
-        if (lane == 0) {
+        // The whole warp walks the stream and waits on the barriers; one elected lane issues.  Kept this way,
+        // control flow and every descriptor are the same in all lanes, which lets them live in the warp's
+        // uniform registers, where the tensor-core instructions take their operands from.  (With a single lane
+        // in a divergent branch each instruction cost that lane 55 - 80 cycles of operand marshalling, whatever
+        // the instruction's size, and the tensor pipe starved behind it.)  A failed wait does not leave the loop:
+        // it switches off the remaining waits and instructions, and the loop runs out.
+        {
+            const bool leader = elect_one();
             constexpr uint32_t idesc_qk = make_idesc(2 * kBlockM, kBlockN, false);
             constexpr uint32_t idesc_pv = make_idesc(2 * kBlockM, D, true);
             bool ok = mbar_wait(q_full, 0, abort_flag, status, 54);
@@ -771,70 +784,78 @@ sa_merge_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             const uint32_t k_empty1 = mapa(smem_u32(k_empty), 1), v_empty1 = mapa(smem_u32(v_empty), 1);
             int pending[2] = {-1, -1};
             int n_done[2] = {0, 0};
-            auto issue_pv = [&](int x, int ip) -> bool {
+            auto wait = [&](uint64_t *bar, int parity, int where) {
+                if (ok) ok = mbar_wait(bar, (uint32_t)parity, abort_flag, status, where);
+            };
+            auto issue_pv = [&](int x, int ip) {
                 const int vs = ip % P::kVStages;
-                if (!mbar_wait(v_full + vs, (ip / P::kVStages) & 1, abort_flag, status, 56)) return false;
-                if (!mbar_wait(p_half + 2 * x, n_done[x] & 1, abort_flag, status, 55)) return false;
+                wait(v_full + vs, (ip / P::kVStages) & 1, 56);
+                wait(p_half + 2 * x, n_done[x] & 1, 55);
                 tc_fence_after();
                 const uint32_t v_lo = v_lo0 + vs * (P::kVHalf >> 4);
                 const uint32_t d_o = tmem_base + col_o(x), a_p = tmem_base + col_s(x);
+                const uint32_t acc0 = n_done[x] > 0 ? 1u : 0u;
+                if (leader && ok) {
+                    mma_ts_lo_pair<idesc_pv>(d_o, a_p, v_lo, acc0);
 #pragma unroll
-                for (int k = 0; k < kBlockN / 32; ++k)
-                    mma_ts_lo_pair<idesc_pv>(d_o, a_p + k * 8, v_lo + k * (16 * 128 >> 4), (n_done[x] > 0 || k > 0) ? 1u : 0u);
-                if (!mbar_wait(p_half + 2 * x + 1, n_done[x] & 1, abort_flag, status, 55)) return false;
+                    for (int k = 1; k < kBlockN / 32; ++k)
+                        mma_ts_lo_pair<idesc_pv>(d_o, a_p + k * 8, v_lo + k * (16 * 128 >> 4), 1u);
+                }
+                wait(p_half + 2 * x + 1, n_done[x] & 1, 55);
                 tc_fence_after();
+                if (leader && ok) {
 #pragma unroll
-                for (int k = kBlockN / 32; k < kBlockN / 16; ++k)
-                    mma_ts_lo_pair<idesc_pv>(d_o, a_p + k * 8, v_lo + k * (16 * 128 >> 4), 1u);
+                    for (int k = kBlockN / 32; k < kBlockN / 16; ++k)
+                        mma_ts_lo_pair<idesc_pv>(d_o, a_p + k * 8, v_lo + k * (16 * 128 >> 4), 1u);
+                }
                 ++n_done[x];
-                return true;
             };
-            for (int i = 0; i < st.n_tiles && ok; ++i) {
+            for (int i = 0; i < st.n_tiles; ++i) {
                 const int ks = i % P::kKStages;
-                ok = mbar_wait(k_full + ks, (i / P::kKStages) & 1, abort_flag, status, 57);
-                if (!ok) break;
+                wait(k_full + ks, (i / P::kKStages) & 1, 57);
                 tc_fence_after();
                 const uint32_t k_lo = k_lo0 + ks * (P::kKHalf >> 4);
-                for (int x = 0; x < 2 && ok; ++x) {
+#pragma unroll
+                for (int x = 0; x < 2; ++x) {
                     const bool present = (x == 0) || st.has_b;
                     if (present && st.used_by(x, i)) {
                         if (pending[x] >= 0) {
                             const int ip = pending[x];
-                            ok = issue_pv(x, ip);
-                            if (!ok) break;
+                            issue_pv(x, ip);
                             // a V stage is released by two arrivals per CTA: pay the other tile's share if it skipped ip
-                            if (!(((1 - x) == 0 || st.has_b) && st.used_by(1 - x, ip))) {
+                            if (leader && ok && !(((1 - x) == 0 || st.has_b) && st.used_by(1 - x, ip))) {
                                 mbar_arrive(v_empty + ip % P::kVStages);
                                 mbar_arrive_cluster(v_empty1 + (ip % P::kVStages) * 8);
                             }
                         }
                         const uint32_t q_lo = q_lo0 + x * (P::kQTile >> 4), d_s = tmem_base + col_s(x);
-                        mma_ss_lo_pair<idesc_qk, 0>(d_s, q_lo, k_lo);
+                        if (leader && ok) {
+                            mma_ss_lo_pair<idesc_qk, 0>(d_s, q_lo, k_lo);
 #pragma unroll
-                        for (int k = 1; k < D / 16; ++k) {
-                            // k-step of 16 elements: 32 bytes within a 64-element swizzle atom; atoms are 128 rows
-                            // apart in a Q tile, 64 rows apart in a CTA's half of a K tile
-                            const uint32_t off_q = ((k / 4) * (kBlockM * 128) + (k % 4) * 32) >> 4;
-                            const uint32_t off_k = ((k / 4) * ((kBlockN / 2) * 128) + (k % 4) * 32) >> 4;
-                            mma_ss_lo_pair<idesc_qk, 1>(d_s, q_lo + off_q, k_lo + off_k);
+                            for (int k = 1; k < D / 16; ++k) {
+                                // k-step of 16 elements: 32 bytes within a 64-element swizzle atom; atoms are 128
+                                // rows apart in a Q tile, 64 rows apart in a CTA's half of a K tile
+                                const uint32_t off_q = ((k / 4) * (kBlockM * 128) + (k % 4) * 32) >> 4;
+                                const uint32_t off_k = ((k / 4) * ((kBlockN / 2) * 128) + (k % 4) * 32) >> 4;
+                                mma_ss_lo_pair<idesc_qk, 1>(d_s, q_lo + off_q, k_lo + off_k);
+                            }
+                            tc_commit_pair(s_full + x, 3);
                         }
-                        tc_commit_pair(s_full + x, 3);
                         pending[x] = i;
-                    } else {
+                    } else if (leader && ok) {
                         mbar_arrive(k_empty + ks);  // the share of a tile that skips this stream tile, in both CTAs
                         mbar_arrive_cluster(k_empty1 + ks * 8);
                     }
                 }
             }
-            for (int x = 0; x < 2 && ok; ++x) {
+#pragma unroll
+            for (int x = 0; x < 2; ++x) {
                 if (pending[x] >= 0) {
-                    const int ip = pending[x];
-                    ok = issue_pv(x, ip);
-                    if (!ok) break;
-                    tc_commit_pair(o_final + x, 3);
+                    issue_pv(x, pending[x]);
+                    if (leader && ok) tc_commit_pair(o_final + x, 3);
                 }
             }
-            if (!ok) {  // no MMA may still be running when tensor memory is freed
+            if (!__all_sync(0xffffffffu, ok) && leader) {  // no MMA may still be running when tensor memory is freed
                 tell_peer();
                 tc_commit_pair_local(drain);
                 mbar_wait_drain(drain, 0);
@@ -845,7 +866,7 @@ sa_merge_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         reg_inc<216>();
         // ------------------------------------------------------------ softmax + epilogue (both CTAs)
         const int x = (warp - 4) >> 2;                 // 0: tile A, 1: tile B
-        softmax_role<D, P::kKStages, P::kVStages, true>(st, x, R0 + x * 2 * kBlockM + (int)rank * kBlockM, tmem_base, s_full,
+        softmax_role<D, P::kKStages, P::kVStages, true, STILL_POLY_OF4>(st, x, R0 + x * 2 * kBlockM + (int)rank * kBlockM, tmem_base, s_full,
                                                         k_empty, v_empty, p_half, mapa(smem_u32(p_half), 0), o_final,
                                                         abort_flag, status, smem + P::kQ + x * P::kQTile, y_part, d_part, n_parts,
                                                         (long long)gridDim.y * N * D, (long long)gridDim.y * N, Y, bh, N, C, lam,

@@ -40,6 +40,16 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
+// One lane of a converged warp (the same lane every time).
+__device__ __forceinline__ bool elect_one() {
+    uint32_t is_leader;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "elect.sync _|p, 0xffffffff;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(is_leader));
+    return is_leader != 0;
+}
 // Bounded wait.  Returns false (and flags the CTA as aborted) when `limit_cycles` have passed
 // or another role has already aborted; `where` goes into the detail word of the status block.
 __device__ __forceinline__ bool mbar_wait_limit(uint64_t *bar, uint32_t parity, volatile int *abort_flag,
@@ -290,6 +300,25 @@ __device__ __forceinline__ float ex2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
+}
+// 2^x for two values on the FMA pipes (x <= 100 or so): n = round(x) through the 1.5 * 2^23 trick, f = x - n in
+// [-1/2, 1/2], 2^f from a cubic (relative error 7.5e-5, a sixtieth of a bf16 rounding step), and n added into
+// the exponent field.  Arguments below -126 (masked columns arrive as -inf) give 2^-126, which is zero in every
+// use made of the result.
+__device__ __forceinline__ float2 exp2_fma2(float2 x) {
+    const float kMagic = 12582912.f;
+    x.x = fmaxf(x.x, -126.f);
+    x.y = fmaxf(x.y, -126.f);
+    const float2 magic = make_float2(kMagic, kMagic);
+    const float2 t = __fadd2_rn(x, magic);
+    const float2 n = __fadd2_rn(t, make_float2(-kMagic, -kMagic));
+    const float2 f = __fadd2_rn(x, make_float2(-n.x, -n.y));
+    float2 p = __ffma2_rn(f, make_float2(0.055171459913253784f, 0.055171459913253784f),
+                          make_float2(0.2426108568906784f, 0.2426108568906784f));
+    p = __ffma2_rn(p, f, make_float2(0.6932609677314758f, 0.6932609677314758f));
+    p = __ffma2_rn(p, f, make_float2(0.9999281167984009f, 0.9999281167984009f));
+    return make_float2(__int_as_float(__float_as_int(p.x) + (__float_as_int(t.x) << 23)),
+                       __int_as_float(__float_as_int(p.y) + (__float_as_int(t.y) << 23)));
 }
 __device__ __forceinline__ float max3(float a, float b, float c) {
     float d;
