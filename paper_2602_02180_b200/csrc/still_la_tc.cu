@@ -377,7 +377,7 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + P::oMisc + 8);
     float *dinv_ring = reinterpret_cast<float *>(smem + P::oDinv);
 
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;   // (known to be the same in all lanes)
     const int bh = blockIdx.x, b = bh / H, h = bh % H, kvh = h / (H / Hkv);
     const int half = blockIdx.y;                // 0: features softmax(u), 1: features softmax(-u)
     const int sc = C / 64;                      // 64-token sub-chunks per chunk
@@ -437,7 +437,7 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem_base = *tmem_base_slot;
+    const uint32_t tmem_base = __shfl_sync(0xffffffffu, *tmem_base_slot, 0);
     // TMEM columns: S^T half [value lanes x d_f features] fp32; f = x W_q of a block [128 rows x d_f]; two read-out
     // results [value lanes x 64 tokens]
     constexpr uint32_t col_state = 0, col_f = DF, col_out = 2 * DF;
@@ -501,81 +501,90 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        // The whole warp walks the schedule and waits on the barriers; one elected lane issues (control flow and
+        // descriptors stay the same in all lanes and can live in uniform registers, where the tensor-core
+        // instructions take their operands from).  A failed wait does not leave the loops: it switches off the
+        // remaining waits and instructions, and the loops run out.
+        {
+            const bool leader = elect_one();
             constexpr uint32_t idesc_f = make_idesc(128, DF, true);
             constexpr uint32_t idesc_upd = make_idesc(128, DF, true) | (1u << 15);  // A M-major, B MN-major
             constexpr uint32_t idesc_rd = make_idesc_tf32(128, 64);
             bool ok = true;
             int nu = 0, nq = 0, nx = 0;
-            // descriptors as low words: a k-step adds a constant (keeps this thread's instruction count low)
+            auto wait = [&](uint64_t *bar, int parity, int where) {
+                if (ok) ok = mbar_wait(bar, (uint32_t)parity, abort_flag, status, where);
+            };
+            // descriptors as low words: a k-step adds a constant
             const uint32_t x_lo = desc_lo(smem_u32(smem + P::oX), 0), w_lo = desc_lo(smem_u32(smem + P::oW), D * 128);
             const uint32_t q_lo0 = desc_lo(smem_u32(smem + P::oQ), 0);
             const uint32_t pk_lo0 = desc_lo(smem_u32(smem + P::oU), 64 * 128);
             const uint32_t v_lo0 = desc_lo(smem_u32(smem + P::oU + P::kPhiK), D == 128 ? 64 * 128 : 0);
             // f = x W_q of block b_first + nx (the map warps have taken the previous f out of tensor memory)
-            auto issue_f = [&]() -> bool {
-                if (nx == 0 && !mbar_wait(w_full, 0, abort_flag, status, 61)) return false;
-                if (!mbar_wait(x_full, nx & 1, abort_flag, status, 62)) return false;
-                if (!mbar_wait(f_free, (nx & 1) ^ 1, abort_flag, status, 63)) return false;
+            auto issue_f = [&]() {
+                if (nx == 0) wait(w_full, 0, 61);
+                wait(x_full, nx & 1, 62);
+                wait(f_free, (nx & 1) ^ 1, 63);
                 tc_fence_after();
+                if (leader && ok) {
 #pragma unroll
-                for (int k = 0; k < D / 16; ++k) {
-                    const uint32_t xo = ((k / 4) * (128 * 128) + (k % 4) * 32) >> 4, wo = (k * (16 * 128)) >> 4;
-                    if (k == 0) mma_ss_lo<idesc_f, 0>(tmem_base + col_f, x_lo + xo, w_lo + wo);
-                    else mma_ss_lo<idesc_f, 1>(tmem_base + col_f, x_lo + xo, w_lo + wo);
+                    for (int k = 0; k < D / 16; ++k) {
+                        const uint32_t xo = ((k / 4) * (128 * 128) + (k % 4) * 32) >> 4, wo = (k * (16 * 128)) >> 4;
+                        if (k == 0) mma_ss_lo<idesc_f, 0>(tmem_base + col_f, x_lo + xo, w_lo + wo);
+                        else mma_ss_lo<idesc_f, 1>(tmem_base + col_f, x_lo + xo, w_lo + wo);
+                    }
+                    tc_commit(f_done);
+                    tc_commit(x_empty);
                 }
-                tc_commit(f_done);
-                tc_commit(x_empty);
                 ++nx;
-                return true;
             };
             if (has_init) {   // the workers have put the sum of the earlier segments into tensor memory
-                ok = mbar_wait(init_done, 0, abort_flag, status, 73);
+                wait(init_done, 0, 73);
                 tc_fence_after();
             }
-            auto issue_update = [&]() -> bool {
-                if (!mbar_wait(u_masked + (nu & 1), (nu >> 1) & 1, abort_flag, status, 64)) return false;
+            auto issue_update = [&]() {
+                wait(u_masked + (nu & 1), (nu >> 1) & 1, 64);
                 tc_fence_after();
                 const uint32_t so = (uint32_t)(nu & 1) * (P::kUStage >> 4);
+                const uint32_t acc0 = (nu > 0 || has_init) ? 1u : 0u;
+                if (leader && ok) {
+                    mma_ss_lo_acc<idesc_upd>(tmem_base + col_state, v_lo0 + so, pk_lo0 + so, acc0);
 #pragma unroll
-                for (int k = 0; k < 4; ++k)   // 16 tokens per step: 16 rows of 128 bytes in both operands
-                    mma_ss_lo_acc<idesc_upd>(tmem_base + col_state, v_lo0 + so + k * (2048 >> 4), pk_lo0 + so + k * (2048 >> 4),
-                                             (nu > 0 || k > 0 || has_init) ? 1u : 0u);
-                tc_commit(u_empty + (nu & 1));
+                    for (int k = 1; k < 4; ++k)   // 16 tokens per step: 16 rows of 128 bytes in both operands
+                        mma_ss_lo_acc<idesc_upd>(tmem_base + col_state, v_lo0 + so + k * (2048 >> 4), pk_lo0 + so + k * (2048 >> 4), 1u);
+                    tc_commit(u_empty + (nu & 1));
+                }
                 ++nu;
-                return true;
             };
             if (sums_only)
-                while (ok && nu < n_upd) ok = issue_update();
-            if (ok && NB > b_first) ok = issue_f();
-            for (int u = u_first; u < NU && ok && !sums_only; ++u) {
+                while (nu < n_upd) issue_update();
+            if (NB > b_first) issue_f();
+            for (int u = u_first; u < NU && !sums_only; ++u) {
                 if (u % sc == 0) {
                     // the chunk that has just left the local region: sub-chunks of chunk u / sc - 2
-                    for (int j = 0; j < per_chunk && ok; ++j) ok = issue_update();
-                    if (!ok) break;
+                    for (int j = 0; j < per_chunk; ++j) issue_update();
                 }
-                ok = mbar_wait(pq_full + (u & 1), (nq >> 1) & 1, abort_flag, status, 65);
-                if (ok) ok = mbar_wait(out_free + (nq & 1), ((nq >> 1) & 1) ^ 1, abort_flag, status, 66);
-                if (!ok) break;
+                wait(pq_full + (u & 1), (nq >> 1) & 1, 65);
+                wait(out_free + (nq & 1), ((nq >> 1) & 1) ^ 1, 66);
                 tc_fence_after();
                 const uint32_t q_lo = q_lo0 + (uint32_t)(u & 1) * (P::kPhiQ >> 4), d_out_t = tmem_base + col_out + (nq & 1) * 64;
+                if (leader && ok) {
 #pragma unroll
-                for (int k = 0; k < DF / 8; ++k) {   // 8 features per step: 32 bytes within a 32-feature atom
-                    const uint32_t qo = ((k / 4) * (64 * 128) + (k % 4) * 32) >> 4;
-                    if (k == 0) mma_ts_tf32_lo<idesc_rd, 0>(d_out_t, tmem_base + col_state, q_lo + qo);
-                    else mma_ts_tf32_lo<idesc_rd, 1>(d_out_t, tmem_base + col_state + k * 8, q_lo + qo);
+                    for (int k = 0; k < DF / 8; ++k) {   // 8 features per step: 32 bytes within a 32-feature atom
+                        const uint32_t qo = ((k / 4) * (64 * 128) + (k % 4) * 32) >> 4;
+                        if (k == 0) mma_ts_tf32_lo<idesc_rd, 0>(d_out_t, tmem_base + col_state, q_lo + qo);
+                        else mma_ts_tf32_lo<idesc_rd, 1>(d_out_t, tmem_base + col_state + k * 8, q_lo + qo);
+                    }
+                    tc_commit(r_done + (nq & 1));
+                    tc_commit(pq_empty + (u & 1));
                 }
-                tc_commit(r_done + (nq & 1));
-                tc_commit(pq_empty + (u & 1));
                 ++nq;
                 // the next block's f while this block's second sub-chunk is read out
-                if ((u & 1) == 0 && b_first + nx < NB) ok = issue_f();
+                if ((u & 1) == 0 && b_first + nx < NB) issue_f();
             }
-            if (ok) tc_commit(fin);   // state after the last update, for the decode state
-            if (!ok) {
-                tc_commit(fin);
-                mbar_wait_drain(fin, 0);
-            }
+            // state after the last update, for the decode state; after a failure, nothing issued may still run
+            if (leader) tc_commit(fin);
+            if (!__all_sync(0xffffffffu, ok) && leader) mbar_wait_drain(fin, 0);
         }
     } else if (warp == 2) {
         // ------------------------------------------------------------ mask warp

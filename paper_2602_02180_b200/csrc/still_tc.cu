@@ -42,6 +42,8 @@
 #include "still_common.cuh"
 #include "still_tc_ptx.cuh"
 
+// Column pairs out of every four whose exponential is computed on the FMA pipes (see softmax_role); measured
+// best at one: two and three were slower on both head dims.
 #ifndef STILL_POLY_OF4
 #define STILL_POLY_OF4 1
 #endif
@@ -356,7 +358,7 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     uint32_t *tmem_base_slot = reinterpret_cast<uint32_t *>(smem + P::kMisc);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + P::kMisc + 8);
 
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;   // (known to be the same in all lanes)
     const int qb = n_qblocks - 1 - blockIdx.x;  // heavy blocks first
     const int bh = blockIdx.y, b = bh / H, h = bh % H, kvh = h / (H / Hkv);
     const int R0 = qb * 2 * kBlockM;
@@ -395,7 +397,7 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem_base = *tmem_base_slot;
+    const uint32_t tmem_base = __shfl_sync(0xffffffffu, *tmem_base_slot, 0);
     // TMEM columns: S_A [0,128), S_B [128,256), O_A [256,256+D), O_B [256+D, 256+2D); P_X overlays S_X.
     auto col_s = [](int x) -> uint32_t { return (uint32_t)x * 128u; };
     auto col_o = [](int x) -> uint32_t { return 256u + (uint32_t)x * (uint32_t)D; };
@@ -475,76 +477,90 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        // The whole warp walks the stream and waits on the barriers; one elected lane issues (control flow and
+        // descriptors stay the same in all lanes and can live in uniform registers, where the tensor-core
+        // instructions take their operands from).  A failed wait does not leave the loop: it switches off the
+        // remaining waits and instructions, and the loop runs out.
+        {
+            const bool leader = elect_one();
             constexpr uint32_t idesc_qk = make_idesc(kBlockM, kBlockN, false);
             constexpr uint32_t idesc_pv = make_idesc(kBlockM, D, true);
             bool ok = mbar_wait(q_full, 0, abort_flag, status, 4);
             tc_fence_after();
-            // descriptors as low words: a k-step adds a constant (keeps this thread's instruction count low)
+            // descriptors as low words: a k-step adds a constant
             const uint32_t q_lo0 = desc_lo(smem_u32(smem + P::kQ), 0);
             const uint32_t k_lo0 = desc_lo(smem_u32(smem + P::kK), 0);
             const uint32_t v_lo0 = desc_lo(smem_u32(smem + P::kV), kBlockN * 128);
             int pending[2] = {-1, -1};   // stream tile whose P V product is still to be issued
             int n_done[2] = {0, 0};      // tiles processed per query tile (phase of p_full)
-            auto issue_pv = [&](int x, int ip) -> bool {
+            auto wait = [&](uint64_t *bar, int parity, int where) {
+                if (ok) ok = mbar_wait(bar, (uint32_t)parity, abort_flag, status, where);
+            };
+            auto issue_pv = [&](int x, int ip) {
                 const int vs = ip % P::kVStages;
                 // (V has normally arrived long ago: checking it first hides the check behind the wait for P)
-                if (!mbar_wait(v_full + vs, (ip / P::kVStages) & 1, abort_flag, status, 6)) return false;
-                if (!mbar_wait(p_half + 2 * x, n_done[x] & 1, abort_flag, status, 5)) return false;
+                wait(v_full + vs, (ip / P::kVStages) & 1, 6);
+                wait(p_half + 2 * x, n_done[x] & 1, 5);
                 tc_fence_after();
                 const uint32_t v_lo = v_lo0 + vs * (P::kTileBytes >> 4);
                 const uint32_t d_o = tmem_base + col_o(x), a_p = tmem_base + col_s(x);
+                const uint32_t acc0 = n_done[x] > 0 ? 1u : 0u;
+                if (leader && ok) {
+                    mma_ts_lo<idesc_pv>(d_o, a_p, v_lo, acc0);
 #pragma unroll
-                for (int k = 0; k < kBlockN / 32; ++k)
-                    mma_ts_lo<idesc_pv>(d_o, a_p + k * 8, v_lo + k * (16 * 128 >> 4), (n_done[x] > 0 || k > 0) ? 1u : 0u);
-                if (!mbar_wait(p_half + 2 * x + 1, n_done[x] & 1, abort_flag, status, 5)) return false;
+                    for (int k = 1; k < kBlockN / 32; ++k)
+                        mma_ts_lo<idesc_pv>(d_o, a_p + k * 8, v_lo + k * (16 * 128 >> 4), 1u);
+                }
+                wait(p_half + 2 * x + 1, n_done[x] & 1, 5);
                 tc_fence_after();
+                if (leader && ok) {
 #pragma unroll
-                for (int k = kBlockN / 32; k < kBlockN / 16; ++k)
-                    mma_ts_lo<idesc_pv>(d_o, a_p + k * 8, v_lo + k * (16 * 128 >> 4), 1u);
+                    for (int k = kBlockN / 32; k < kBlockN / 16; ++k)
+                        mma_ts_lo<idesc_pv>(d_o, a_p + k * 8, v_lo + k * (16 * 128 >> 4), 1u);
+                }
                 ++n_done[x];
-                return true;
             };
-            for (int i = 0; i < st.n_tiles && ok; ++i) {
+            for (int i = 0; i < st.n_tiles; ++i) {
                 const int ks = i % P::kKStages;
-                ok = mbar_wait(k_full + ks, (i / P::kKStages) & 1, abort_flag, status, 7);
-                if (!ok) break;
+                wait(k_full + ks, (i / P::kKStages) & 1, 7);
                 tc_fence_after();
                 const uint32_t k_lo = k_lo0 + ks * (P::kTileBytes >> 4);
-                for (int x = 0; x < 2 && ok; ++x) {
+#pragma unroll
+                for (int x = 0; x < 2; ++x) {
                     const bool present = (x == 0) || st.has_b;
                     if (present && st.used_by(x, i)) {
                         if (pending[x] >= 0) {
                             const int ip = pending[x];
-                            ok = issue_pv(x, ip);
-                            if (!ok) break;
+                            issue_pv(x, ip);
                             // a V stage is released by two arrivals: pay the other tile's share if it skipped ip
-                            if (!(((1 - x) == 0 || st.has_b) && st.used_by(1 - x, ip))) mbar_arrive(v_empty + ip % P::kVStages);
+                            if (leader && ok && !(((1 - x) == 0 || st.has_b) && st.used_by(1 - x, ip)))
+                                mbar_arrive(v_empty + ip % P::kVStages);
                         }
                         const uint32_t q_lo = q_lo0 + x * (P::kTileBytes >> 4), d_s = tmem_base + col_s(x);
-                        mma_ss_lo<idesc_qk, 0>(d_s, q_lo, k_lo);
+                        if (leader && ok) {
+                            mma_ss_lo<idesc_qk, 0>(d_s, q_lo, k_lo);
 #pragma unroll
-                        for (int k = 1; k < D / 16; ++k) {
-                            // k-step of 16 elements: 32 bytes within a 64-element swizzle atom, atoms 128 rows apart
-                            const uint32_t off = ((k / 4) * (kBlockM * 128) + (k % 4) * 32) >> 4;
-                            mma_ss_lo<idesc_qk, 1>(d_s, q_lo + off, k_lo + off);
+                            for (int k = 1; k < D / 16; ++k) {
+                                // k-step of 16 elements: 32 bytes within a 64-element swizzle atom, atoms 128 rows apart
+                                const uint32_t off = ((k / 4) * (kBlockM * 128) + (k % 4) * 32) >> 4;
+                                mma_ss_lo<idesc_qk, 1>(d_s, q_lo + off, k_lo + off);
+                            }
+                            tc_commit(s_full + x);
                         }
-                        tc_commit(s_full + x);
                         pending[x] = i;
-                    } else {
+                    } else if (leader && ok) {
                         mbar_arrive(k_empty + ks);  // the share of a tile that skips this stream tile
                     }
                 }
             }
-            for (int x = 0; x < 2 && ok; ++x) {
+#pragma unroll
+            for (int x = 0; x < 2; ++x) {
                 if (pending[x] >= 0) {
-                    const int ip = pending[x];
-                    ok = issue_pv(x, ip);
-                    if (!ok) break;
-                    tc_commit(o_final + x);
+                    issue_pv(x, pending[x]);
+                    if (leader && ok) tc_commit(o_final + x);
                 }
             }
-            if (!ok) {  // no MMA may still be running when tensor memory is freed
+            if (!__all_sync(0xffffffffu, ok) && leader) {  // no MMA may still be running when tensor memory is freed
                 tc_commit(drain);
                 mbar_wait_drain(drain, 0);
             }
@@ -554,7 +570,7 @@ sa_merge_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         reg_inc<216>();
         // ------------------------------------------------------------ softmax + epilogue
         const int x = (warp - 4) >> 2;                 // 0: tile A, 1: tile B
-        softmax_role<D, P::kKStages, P::kVStages, false, 0>(st, x, R0 + x * kBlockM, tmem_base, s_full, k_empty, v_empty, p_half, 0u,
+        softmax_role<D, P::kKStages, P::kVStages, false, STILL_POLY_OF4>(st, x, R0 + x * kBlockM, tmem_base, s_full, k_empty, v_empty, p_half, 0u,
                                                          o_final, abort_flag, status, smem + P::kQ + x * P::kTileBytes, y_part,
                                                          d_part, n_parts, (long long)gridDim.y * N * D, (long long)gridDim.y * N,
                                                          Y, bh, N, C, lam, budget, scale_log2);
