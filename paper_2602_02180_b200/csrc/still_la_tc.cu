@@ -564,6 +564,10 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     // the chunk that has just left the local region: sub-chunks of chunk u / sc - 2
                     for (int j = 0; j < per_chunk; ++j) issue_update();
                 }
+                // The next block's f = x W_q goes out as soon as its rows have arrived and the map warps have taken the
+                // current f out of tensor memory: it is then ready when they finish the current block.  (Issued after
+                // this block's read-out, it made the map warps wait for a round trip through this warp per block.)
+                if ((u & 1) == 0 && b_first + nx < NB) issue_f();
                 wait(pq_full + (u & 1), (nq >> 1) & 1, 65);
                 wait(out_free + (nq & 1), ((nq >> 1) & 1) ^ 1, 66);
                 tc_fence_after();
@@ -579,8 +583,6 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     tc_commit(pq_empty + (u & 1));
                 }
                 ++nq;
-                // the next block's f while this block's second sub-chunk is read out
-                if ((u & 1) == 0 && b_first + nx < NB) issue_f();
             }
             // state after the last update, for the decode state; after a failure, nothing issued may still run
             if (leader) tc_commit(fin);
@@ -812,18 +814,32 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             if (lane == 0) mbar_arrive(f_free);
             float sgn = 0.f, shift = 0.f;
             if (ok) {
-                // (four independent chains each: the row is long and these are latency-bound reductions; this CTA's
-                // half needs only one extremum: max f for softmax(u), min f for softmax(-u))
-                float n2[4] = {0.f, 0.f, 0.f, 0.f}, ex[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-                const float unit = half == 0 ? 1.f : -1.f;
+                // (packed arithmetic and four independent chains each: the row is long and these are latency-bound
+                // reductions; this CTA's half needs only one extremum: max f for softmax(u), min f for softmax(-u))
+                if (bias != nullptr) {
 #pragma unroll
-                for (int j = 0; j < DF; ++j) {
-                    if (bias != nullptr) fv[j] += __bfloat162float(bias[j]);
-                    n2[j & 3] = fmaf(fv[j], fv[j], n2[j & 3]);
-                    ex[j & 3] = fmaxf(ex[j & 3], fv[j] * unit);
+                    for (int j = 0; j < DF; ++j) fv[j] += __bfloat162float(bias[j]);
                 }
-                const float nf2 = (n2[0] + n2[1]) + (n2[2] + n2[3]);
-                const float extreme = fmaxf(fmaxf(ex[0], ex[1]), fmaxf(ex[2], ex[3]));   // max of +-f
+                float2 n2[4];
+                float ex[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    n2[q] = make_float2(0.f, 0.f);
+                    ex[q] = half == 0 ? -INFINITY : INFINITY;
+                }
+#pragma unroll
+                for (int j = 0; j < DF; j += 8) {
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const float2 v = make_float2(fv[j + 2 * q], fv[j + 2 * q + 1]);
+                        n2[q] = __ffma2_rn(v, v, n2[q]);
+                        ex[q] = half == 0 ? max3(ex[q], v.x, v.y) : min3(ex[q], v.x, v.y);
+                    }
+                }
+                const float nf2 = ((n2[0].x + n2[0].y) + (n2[1].x + n2[1].y)) + ((n2[2].x + n2[2].y) + (n2[3].x + n2[3].y));
+                const float unit = half == 0 ? 1.f : -1.f;
+                const float extreme = half == 0 ? fmaxf(fmaxf(ex[0], ex[1]), fmaxf(ex[2], ex[3]))
+                                                : -fminf(fminf(ex[0], ex[1]), fminf(ex[2], ex[3]));   // max of +-f
                 // u = f * ratio in the log2 domain; the exponent of this half is +-u - max(+-u) <= 0
                 const float ratio = sqrtf(nx2) / fmaxf(sqrtf(nf2), 1e-12f) * 1.4426950408889634f;
                 sgn = unit * ratio;
@@ -839,7 +855,8 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 // row is written as it is computed.  The z values of the next group of 16 features are loaded before
                 // the stores of this group (shared-memory loads are kept behind earlier stores).
                 uint8_t *tile = smem + P::oQ + slot * P::kPhiQ;
-                float zs4[4] = {0.f, 0.f, 0.f, 0.f}, ds4[4] = {0.f, 0.f, 0.f, 0.f};
+                float2 zs2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)}, ds2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+                const float2 sgn2 = make_float2(sgn, sgn), shift2 = make_float2(shift, shift);
                 float4 zc[4];
 #pragma unroll
                 for (int i = 0; i < 4; ++i) zc[i] = *reinterpret_cast<const float4 *>(zs + 4 * i);
@@ -852,23 +869,24 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         const int j = 16 * g + 4 * i;
+                        const float2 a0 = __ffma2_rn(make_float2(fv[j], fv[j + 1]), sgn2, shift2);
+                        const float2 a1 = __ffma2_rn(make_float2(fv[j + 2], fv[j + 3]), sgn2, shift2);
                         float4 ev;
-                        ev.x = ex2(fmaf(fv[j], sgn, shift));
-                        ev.y = ex2(fmaf(fv[j + 1], sgn, shift));
-                        ev.z = ex2(fmaf(fv[j + 2], sgn, shift));
-                        ev.w = ex2(fmaf(fv[j + 3], sgn, shift));
-                        zs4[0] += ev.x; zs4[1] += ev.y; zs4[2] += ev.z; zs4[3] += ev.w;
-                        ds4[0] = fmaf(ev.x, zc[i].x, ds4[0]);
-                        ds4[1] = fmaf(ev.y, zc[i].y, ds4[1]);
-                        ds4[2] = fmaf(ev.z, zc[i].z, ds4[2]);
-                        ds4[3] = fmaf(ev.w, zc[i].w, ds4[3]);
+                        ev.x = ex2(a0.x);
+                        ev.y = ex2(a0.y);
+                        ev.z = ex2(a1.x);
+                        ev.w = ex2(a1.y);
+                        zs2[0] = __fadd2_rn(zs2[0], make_float2(ev.x, ev.y));
+                        zs2[1] = __fadd2_rn(zs2[1], make_float2(ev.z, ev.w));
+                        ds2[0] = __ffma2_rn(make_float2(ev.x, ev.y), make_float2(zc[i].x, zc[i].y), ds2[0]);
+                        ds2[1] = __ffma2_rn(make_float2(ev.z, ev.w), make_float2(zc[i].z, zc[i].w), ds2[1]);
                         // features j .. j+3: atom j / 32, 16-byte piece (j % 32) / 4, swizzled by the row
                         *reinterpret_cast<float4 *>(tile + (j >> 5) * (64 * 128) + rr * 128 + ((((j & 31) >> 2) ^ (rr & 7)) << 4)) = ev;
                     }
 #pragma unroll
                     for (int i = 0; i < 4; ++i) zc[i] = zn[i];
                 }
-                const float zsum = (zs4[0] + zs4[1]) + (zs4[2] + zs4[3]), draw = (ds4[0] + ds4[1]) + (ds4[2] + ds4[3]);
+                const float zsum = (zs2[0].x + zs2[0].y) + (zs2[1].x + zs2[1].y), draw = (ds2[0].x + ds2[0].y) + (ds2[1].x + ds2[1].y);
                 const int t = u * 64 + rr;
                 if (t < N) d_out[(long long)bh * N + t] = draw / zsum;     // D_part
                 dinv_ring[(u & 7) * 64 + rr] = draw > 0.f ? 1.f / draw : 0.f;
