@@ -250,6 +250,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c3", choices=["c1", "c2", "c3", "c4", "c5"])
     ap.add_argument("--topk", type=int, default=None, help="override lambda (e.g. the C/4 companion)")
+    ap.add_argument("--max-salient", type=int, default=0, help="salient-cache budget per head (a multiple of topk; 0: none)")
     ap.add_argument("--B", type=int, default=None, help="override the batch (profiling of a smaller case)")
     ap.add_argument("--H", type=int, default=None, help="override the query heads (KV heads scale along)")
     ap.add_argument("--N", type=int, default=None, help="override the sequence length")
@@ -387,14 +388,14 @@ def prefill_companion(name, w, lam, steps, still, synth, torch, dev, max_salient
 
 def bench_prefill(args, w, lam, still, synth, torch, dist, dev, rank, world):
     warmup = max(args.warmup, 10)
-    m = time_prefill(w, lam, args.steps, warmup, still, synth, torch, dist, dev, rank)
+    m = time_prefill(w, lam, args.steps, warmup, still, synth, torch, dist, dev, rank, max_salient=args.max_salient)
     p, Q, K, V, Wq, Wk = m.pop("tensors")
     ms_total = _max_over_ranks(torch, dist, m["ms_total"], dev)
     kernel_ms, clocks, launches_per_step = m["kernel_ms"], m["clocks"], m["launches_per_step"]
     ms_step = ms_total / args.steps
     value = world * w.B * w.N / (ms_step * 1e-3)
 
-    work = algorithmic_work(w, lam)
+    work = algorithmic_work(w, lam, args.max_salient)
     peaks = measured_peaks()
     nominal, measured = roofline_times(work, peaks)
     k_ms = statistics.mean(kernel_ms) if kernel_ms else None
@@ -480,7 +481,7 @@ def bench_prefill(args, w, lam, still, synth, torch, dist, dev, rank, world):
         "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16" if not fp32 else "f32", "data": "synthetic",
         "config": {"workload": w.name, "B": w.B, "H": w.H, "Hkv": w.Hkv, "d": w.d, "N": w.N, "chunk": w.C,
-                   "topk": lam, "l2": "inputs larger than L2 (no flush)", "per_gpu_batch": w.B,
+                   "topk": lam, "max_salient": args.max_salient, "l2": "inputs larger than L2 (no flush)", "per_gpu_batch": w.B,
                    "timing": "K steps bracketed by one CUDA-event pair (ms_per_step, value); every step also has its own "
                              "pair (ms_per_step_median)"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
@@ -570,13 +571,14 @@ def bench_decode(args, w, lam, still, synth, torch, dist, dev, rank, world):
     are timed.  HBM-bound: the salient K/V history is read once per KV head per step."""
     n_steps = args.steps
     warmup = max(args.warmup, 3)
-    m = time_decode(w, lam, n_steps, warmup, still, synth, torch, dist, dev, rank, reserve=64 + w.steps)
+    m = time_decode(w, lam, n_steps, warmup, still, synth, torch, dist, dev, rank, reserve=64 + w.steps,
+                    max_salient=args.max_salient)
     p, state, cap, ins, y, Wq, Wk, wl = m.pop("ctx")
     t, launches, clocks, kernel_ms = m["t"], m["launches"], m["clocks"], m["kernel_ms"]
     ms_total = _max_over_ranks(torch, dist, m["ms_total"], dev)
     ms_step = ms_total / n_steps
     peaks = measured_peaks()
-    by = decode_bytes(w, lam, t)
+    by = decode_bytes(w, lam, t, args.max_salient)
     k_ms = statistics.mean(kernel_ms) if kernel_ms else ms_step
     ach = by / (k_ms * 1e-3) / 1e9
     roof = {"bound": "hbm", "kernel": "split-KV attend", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
@@ -620,7 +622,7 @@ def bench_decode(args, w, lam, still, synth, torch, dist, dev, rank, world):
         "ms_per_step_median": statistics.median(m["per_step"]),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": w.name, "B": w.B, "H": w.H, "Hkv": w.Hkv, "d": w.d, "prefix": w.N, "chunk": w.C,
-                   "topk": lam, "l2": "K/V history larger than L2 (no flush)"},
+                   "topk": lam, "max_salient": args.max_salient, "l2": "K/V history larger than L2 (no flush)"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches * n_steps, "roofline": roof, "cpu_baseline": cpu,
     }
 

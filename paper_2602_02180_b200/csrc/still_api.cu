@@ -87,7 +87,9 @@ static FwdPlan plan_fwd(const still_params_t *p, long long N) {
             // tensor-core branch: phi(Q) is never stored; the branch leaves two bf16 partial results
             w.csum = take(BHkv * (size_t)T * dp * 4);
             w.zpre = take(BH * (size_t)std::max<long long>(T - 2, 1) * dp * 4);
-            w.segs = take(BH * (size_t)std::max(tc_la_segments(p, N, nullptr) - 1, 1) * dp * p->d * 4);
+            int seg_chunks = 0;
+            const int n_seg = tc_la_segments(p, N, &seg_chunks);
+            w.segs = take(BH * (size_t)std::max((n_seg - 1) * tc_la_sum_parts(seg_chunks), 1) * dp * p->d * 4);
         } else {
             w.phiQ = take(BH * (size_t)N * dp * es);
             w.nla = take(BH * (size_t)N * p->d * 4);

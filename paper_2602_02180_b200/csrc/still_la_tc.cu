@@ -339,18 +339,20 @@ struct FusedPlan {
     static constexpr int kW = D * DF * 2;               // W_q, MN-major (as TMA delivers [d rows, d_f columns])
     static constexpr int kX = 128 * D * 2;              // raw Q rows of one block of 128 tokens
     static constexpr int kPhiQ = 64 * DF * 4;           // phi_q half of 64 tokens, fp32 (TF32 operand)
-    static constexpr int kPhiK = 64 * DF * 2;           // phi_k half of 64 tokens, bf16
-    static constexpr int kVt = 64 * D * 2;              // V of 64 tokens
+    static constexpr int kUTok = 32;                    // tokens per state-update tile
+    static constexpr int kUStages = 4;                  // ring of update tiles (loads run this far ahead of the MMAs)
+    static constexpr int kPhiK = kUTok * DF * 2;        // phi_k half of an update tile, bf16
+    static constexpr int kVt = kUTok * D * 2;           // V of an update tile
     static constexpr int kUStage = kPhiK + kVt;
     static constexpr int oW = 0;
     static constexpr int oX = oW + kW;
     static constexpr int oQ = oX + kX;                  // two slots
-    static constexpr int oU = oQ + 2 * kPhiQ;           // two stages
-    static constexpr int oDinv = oU + 2 * kUStage;      // [8][64] 1 / D_part of the tokens of the last sub-chunks
+    static constexpr int oU = oQ + 2 * kPhiQ;           // kUStages stages
+    static constexpr int oDinv = oU + kUStages * kUStage;      // [8][64] 1 / D_part of the tokens of the last sub-chunks
     static constexpr int oZ = oDinv + 8 * 64 * 4;       // [4 map warps][d_f] z half of the chunk two back
     static constexpr int oStage = oZ + 4 * DF * 4;      // [64 tokens][d] bf16: the output of a sub-chunk on its way out
     static constexpr int oBar = oStage + 64 * D * 2;
-    static constexpr int kNumBars = 24;
+    static constexpr int kNumBars = 28;
     static constexpr int oMisc = oBar + kNumBars * 8;
     static constexpr int kTotal = oMisc + 16;
 };
@@ -365,14 +367,15 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 const int32_t *__restrict__ sel_idx, const float *__restrict__ zpre, __nv_bfloat16 *__restrict__ y_part,
                 float *__restrict__ d_part, float *__restrict__ S_out, float *__restrict__ seg_sums, int *status, int H, int Hkv,
                 int N, int C, int lam, int window, long long part_stride_y, long long part_stride_d, int seg_chunks, int n_seg,
-                int sums_only) {
+                int sum_parts, int sums_only) {
     using P = FusedPlan<D, DF>;
     constexpr int NF = 2 * DF;
     extern __shared__ __align__(1024) uint8_t smem[];
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + P::oBar);
     uint64_t *w_full = bars, *x_full = bars + 1, *x_empty = bars + 2, *f_done = bars + 3, *f_free = bars + 4;
-    uint64_t *pq_full = bars + 5, *pq_empty = bars + 7, *u_full = bars + 9, *u_empty = bars + 11, *u_masked = bars + 13;
-    uint64_t *r_done = bars + 15, *out_free = bars + 17, *fin = bars + 19, *init_done = bars + 20;
+    uint64_t *pq_full = bars + 5, *pq_empty = bars + 7, *r_done = bars + 9, *out_free = bars + 11, *fin = bars + 13;
+    uint64_t *init_done = bars + 14, *u_full = bars + 15, *u_empty = u_full + P::kUStages, *u_masked = u_empty + P::kUStages;
+    constexpr int kUS = P::kUStages, kUTok = P::kUTok;
     uint32_t *tmem_base_slot = reinterpret_cast<uint32_t *>(smem + P::oMisc);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + P::oMisc + 8);
     float *dinv_ring = reinterpret_cast<float *>(smem + P::oDinv);
@@ -386,16 +389,20 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     // The sequence is cut into n_seg segments of seg_chunks chunks (two-level scan): segment g answers the
     // sub-chunks [u_first, NU) and performs the updates that fall between them, starting from the sum of the
     // earlier segments' updates (seg_sums, produced by a first pass of this kernel with sums_only set).
+    // The first pass cuts every segment into sum_parts pieces, one CTA each (it has no scan to keep in order, and
+    // the pieces fill the SMs that the n_seg - 1 summed segments alone would leave idle).
     const int seg = blockIdx.z;
+    if (sums_only) seg_chunks /= sum_parts;
     const int NU_all = (N + 63) / 64;           // sub-chunks with query rows
     const int u_first = seg == 0 ? 2 * sc : seg * seg_chunks * sc;   // the first two chunks see an empty state
     const int NU = (!sums_only && seg == n_seg - 1) ? NU_all : min(NU_all, (seg + 1) * seg_chunks * sc);
     const int b_first = u_first / 2;            // blocks of 128 query rows: [b_first, NB)
     const int NB = sums_only ? b_first : (NU + 1) / 2;
-    // Update tiles: per routed chunk its sc sub-chunks (selected rows zeroed) and, with a salient-cache budget of
-    // `window` chunks, the sc sub-chunks of the chunk `window` back with everything but its selected rows zeroed:
-    // those tokens leave the cache for the state when the chunk is routed.
-    const int per_chunk = window > 0 ? 2 * sc : sc;
+    // Update tiles of kUTok tokens: per routed chunk its su tiles (selected rows zeroed) and, with a salient-cache
+    // budget of `window` chunks, the su tiles of the chunk `window` back with everything but its selected rows
+    // zeroed: those tokens leave the cache for the state when the chunk is routed.
+    const int su = C / kUTok;
+    const int per_chunk = window > 0 ? 2 * su : su;
     const int nu0 = (u_first / sc - 2) * per_chunk;    // first update tile of the segment
     const int n_upd = NU > u_first ? ((NU - 1) / sc - 1) * per_chunk - nu0 : 0;
     const bool has_init = !sums_only && seg > 0;
@@ -419,11 +426,13 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         for (int i = 0; i < 2; ++i) {
             mbar_init(pq_full + i, 2);   // the two map warps that own the slot's 64 rows
             mbar_init(pq_empty + i, 1);
+            mbar_init(r_done + i, 1);
+            mbar_init(out_free + i, 4);
+        }
+        for (int i = 0; i < kUS; ++i) {
             mbar_init(u_full + i, 1);
             mbar_init(u_empty + i, 1);
             mbar_init(u_masked + i, 1);
-            mbar_init(r_done + i, 1);
-            mbar_init(out_free + i, 4);
         }
         mbar_init(fin, 1);
         mbar_init(init_done, 4);
@@ -466,18 +475,18 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     ++nx;
                     progressed = true;
                 }
-                if (nu < n_upd && mbar_try_wait(u_empty + (nu & 1), ((nu >> 1) & 1) ^ 1)) {
-                    uint8_t *stg = smem + P::oU + (nu & 1) * P::kUStage;
+                if (nu < n_upd && mbar_try_wait(u_empty + nu % kUS, ((nu / kUS) & 1) ^ 1)) {
+                    uint8_t *stg = smem + P::oU + (nu % kUS) * P::kUStage;
                     // tile a = nu0 + nu: chunk a / per_chunk, then which of its tiles; a leaving-tile reads the chunk
                     // `window` back (before there is one, any valid tile: all its rows are zeroed)
                     const int a_t = nu0 + nu, cc = a_t / per_chunk, rt = a_t % per_chunk;
-                    const int src = (rt >= sc && cc >= window) ? cc - window : cc;
-                    const int tile_sub = src * sc + rt % sc;
-                    mbar_expect_tx(u_full + (nu & 1), P::kUStage);
-                    for (int a = 0; a < DF / 64; ++a)  // phi(K) half: MN-major, 64-feature atoms 64 rows apart
-                        tma_load_2d(stg + a * (64 * 128), &tm_phik, u_full + (nu & 1), half * DF + a * 64, kv_row0 + tile_sub * 64);
-                    for (int a = 0; a < D / 64; ++a)   // V: M-major A operand, 64-column atoms 64 rows apart
-                        tma_load_2d(stg + P::kPhiK + a * (64 * 128), &tm_v, u_full + (nu & 1), a * 64, kv_row0 + tile_sub * 64);
+                    const int src = (rt >= su && cc >= window) ? cc - window : cc;
+                    const int tile_sub = src * su + rt % su;
+                    mbar_expect_tx(u_full + nu % kUS, P::kUStage);
+                    for (int a = 0; a < DF / 64; ++a)  // phi(K) half: MN-major, 64-feature atoms kUTok rows apart
+                        tma_load_2d(stg + a * (kUTok * 128), &tm_phik, u_full + nu % kUS, half * DF + a * 64, kv_row0 + tile_sub * kUTok);
+                    for (int a = 0; a < D / 64; ++a)   // V: M-major A operand, 64-column atoms kUTok rows apart
+                        tma_load_2d(stg + P::kPhiK + a * (kUTok * 128), &tm_v, u_full + nu % kUS, a * 64, kv_row0 + tile_sub * kUTok);
                     ++nu;
                     progressed = true;
                 }
@@ -494,7 +503,7 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 }
             }
             if (*abort_flag) {  // leave no copy in flight behind
-                if (nu > 0) mbar_wait_drain(u_full + ((nu - 1) & 1), ((nu - 1) >> 1) & 1);
+                if (nu > 0) mbar_wait_drain(u_full + (nu - 1) % kUS, ((nu - 1) / kUS) & 1);
                 if (nx > 0) mbar_wait_drain(x_full, (nx - 1) & 1);
                 if (n_blk > 0) mbar_wait_drain(w_full, 0);
             }
@@ -518,8 +527,8 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             // descriptors as low words: a k-step adds a constant
             const uint32_t x_lo = desc_lo(smem_u32(smem + P::oX), 0), w_lo = desc_lo(smem_u32(smem + P::oW), D * 128);
             const uint32_t q_lo0 = desc_lo(smem_u32(smem + P::oQ), 0);
-            const uint32_t pk_lo0 = desc_lo(smem_u32(smem + P::oU), 64 * 128);
-            const uint32_t v_lo0 = desc_lo(smem_u32(smem + P::oU + P::kPhiK), D == 128 ? 64 * 128 : 0);
+            const uint32_t pk_lo0 = desc_lo(smem_u32(smem + P::oU), kUTok * 128);
+            const uint32_t v_lo0 = desc_lo(smem_u32(smem + P::oU + P::kPhiK), D == 128 ? kUTok * 128 : 0);
             // f = x W_q of block b_first + nx (the map warps have taken the previous f out of tensor memory)
             auto issue_f = [&]() {
                 if (nx == 0) wait(w_full, 0, 61);
@@ -543,16 +552,16 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 tc_fence_after();
             }
             auto issue_update = [&]() {
-                wait(u_masked + (nu & 1), (nu >> 1) & 1, 64);
+                wait(u_masked + nu % kUS, (nu / kUS) & 1, 64);
                 tc_fence_after();
-                const uint32_t so = (uint32_t)(nu & 1) * (P::kUStage >> 4);
+                const uint32_t so = (uint32_t)(nu % kUS) * (P::kUStage >> 4);
                 const uint32_t acc0 = (nu > 0 || has_init) ? 1u : 0u;
                 if (leader && ok) {
                     mma_ss_lo_acc<idesc_upd>(tmem_base + col_state, v_lo0 + so, pk_lo0 + so, acc0);
 #pragma unroll
-                    for (int k = 1; k < 4; ++k)   // 16 tokens per step: 16 rows of 128 bytes in both operands
+                    for (int k = 1; k < kUTok / 16; ++k)   // 16 tokens per step: 16 rows of 128 bytes in both operands
                         mma_ss_lo_acc<idesc_upd>(tmem_base + col_state, v_lo0 + so + k * (2048 >> 4), pk_lo0 + so + k * (2048 >> 4), 1u);
-                    tc_commit(u_empty + (nu & 1));
+                    tc_commit(u_empty + nu % kUS);
                 }
                 ++nu;
             };
@@ -588,49 +597,56 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             if (leader) tc_commit(fin);
             if (!__all_sync(0xffffffffu, ok) && leader) mbar_wait_drain(fin, 0);
         }
-    } else if (warp == 2) {
-        // ------------------------------------------------------------ mask warp
+    } else {
+        // ------------------------------------------------------------ mask warps (2 and 3: alternate tiles)
         // Zeroes, in every phi(K) tile, the rows of the tokens kept for softmax attention: only the others enter the
-        // state.  The chunk's indices are fetched before the tile is waited for.
+        // state.  The indices of a tile's chunk are requested one tile ahead (a round trip to L2 per tile would
+        // otherwise pace the whole update path), and two warps take turns.
         bool ok = true;
-        for (int nu = 0; nu < n_upd; ++nu) {
-            const int a_t = nu0 + nu, cc = a_t / per_chunk, rt = a_t % per_chunk, sub = rt % sc;
-            const bool leaving = rt >= sc;                       // tile of the tokens that leave the salient cache
-            const int chunk = leaving ? cc - window : cc;        // (chunk < 0: nothing leaves yet, every row is zeroed)
-            int row[4];
+        // positions of the selected tokens of tile nu's chunk relative to the tile's first row (-1: none)
+        auto fetch = [&](int nu, int (&r)[4]) {
+            const int a_t = nu0 + nu, cc = a_t / per_chunk, rt = a_t % per_chunk, sub = rt % su;
+            const int chunk = rt >= su ? cc - window : cc;       // (chunk < 0: nothing leaves yet, every row is zeroed)
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
                 const int i = lane + 32 * q;
-                row[q] = (i < lam && chunk >= 0) ? sel_idx[((long long)bh * Tn + chunk) * lam + i] - (chunk * C + sub * 64) : -1;
+                r[q] = (nu < n_upd && i < lam && chunk >= 0)
+                           ? sel_idx[((long long)bh * Tn + chunk) * lam + i] - (chunk * C + sub * kUTok) : -1;
             }
-            // the selected rows of the tile as a 64-bit set
-            uint32_t lo = 0u, hi = 0u;
+        };
+        int cur[4], nxt[4];
+        fetch(warp - 2, cur);
+        for (int nu = warp - 2; nu < n_upd; nu += 2) {
+            fetch(nu + 2, nxt);
+            const bool leaving = (nu0 + nu) % per_chunk >= su;   // tile of the tokens that leave the salient cache
+            // the selected rows of the tile as a 32-bit set
+            uint32_t rows = 0u;
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                if (row[q] >= 0 && row[q] < 32) lo |= 1u << row[q];
-                if (row[q] >= 32 && row[q] < 64) hi |= 1u << (row[q] - 32);
-            }
-            lo = __reduce_or_sync(0xffffffffu, lo);
-            hi = __reduce_or_sync(0xffffffffu, hi);
-            if (leaving) { lo = ~lo; hi = ~hi; }                 // rows to zero: the selected ones, or all the others
-            if (ok) ok = mbar_wait(u_full + (nu & 1), (nu >> 1) & 1, abort_flag, status, 67);
+            for (int q = 0; q < 4; ++q)
+                if (cur[q] >= 0 && cur[q] < kUTok) rows |= 1u << cur[q];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) cur[q] = nxt[q];
+            rows = __reduce_or_sync(0xffffffffu, rows);
+            if (leaving) rows = ~rows;                           // rows to zero: the selected ones, or all the others
+            if (ok) ok = mbar_wait(u_full + nu % kUS, (nu / kUS) & 1, abort_flag, status, 67);
             ok = __all_sync(0xffffffffu, ok);
             if (ok) {
-                uint8_t *tile = smem + P::oU + (nu & 1) * P::kUStage;
+                // A row is 128 bytes in each 64-feature atom.  Eight lanes clear one such line (all 32 banks, no
+                // conflict), so a store instruction clears the lines of four rows.
+                uint8_t *tile = smem + P::oU + (nu % kUS) * P::kUStage;
 #pragma unroll
-                for (int hh = 0; hh < 2; ++hh) {                 // lane l looks after rows l and l + 32
-                    if (((hh == 0 ? lo : hi) >> lane) & 1u) {
-                        const int rz = hh * 32 + lane;
+                for (int it = 0; it < kUTok / 4; ++it) {
+                    const int rz = it * 4 + (lane >> 3);
+                    if ((rows >> rz) & 1u) {
 #pragma unroll
-                        for (int piece = 0; piece < DF / 8; ++piece)   // 16-byte pieces of the token's feature half
-                            *reinterpret_cast<uint4 *>(tile + (piece >> 3) * (64 * 128) + rz * 128 + ((piece & 7) << 4)) =
-                                make_uint4(0, 0, 0, 0);
+                        for (int a = 0; a < DF / 64; ++a)
+                            *reinterpret_cast<uint4 *>(tile + a * (kUTok * 128) + rz * 128 + ((lane & 7) << 4)) = make_uint4(0, 0, 0, 0);
                     }
                 }
                 fence_proxy_async();
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(u_masked + (nu & 1));
+            if (lane == 0) mbar_arrive(u_masked + nu % kUS);
         }
     }
     } else if (warp < 8) {
@@ -651,7 +667,8 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
         if (has_init) {
             // S^T of this segment starts as the sum of the earlier segments' updates: lane e, column f <- sum_g P_g[f][e]
-            const float *P0 = seg_sums + (((long long)bh * 2 + half) * (n_seg - 1)) * (DF * D);
+            const float *P0 = seg_sums + (((long long)bh * 2 + half) * ((n_seg - 1) * sum_parts)) * (DF * D);
+            const int n_sums = seg * sum_parts;
 #pragma unroll 1
             for (int q = 0; q < DF / 32; ++q) {
                 uint32_t sreg[32];
@@ -659,7 +676,7 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 for (int j = 0; j < 32; ++j) {
                     float acc = 0.f;
                     if (e < D)
-                        for (int g2 = 0; g2 < seg; ++g2) acc += P0[(long long)g2 * (DF * D) + (q * 32 + j) * D + e];
+                        for (int g2 = 0; g2 < n_sums; ++g2) acc += P0[(long long)g2 * (DF * D) + (q * 32 + j) * D + e];
                     sreg[j] = __float_as_uint(acc);
                 }
                 tmem_st32(taddr + col_state + q * 32, sreg);
@@ -731,7 +748,7 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         // the state after the segment's last update: the segment's own sum for the second pass (sums_only), or,
         // from the last segment, S [2 d_f, d] of the decode state (this CTA's features)
         float *S_dst = nullptr;
-        if (sums_only) S_dst = seg_sums + (((long long)bh * 2 + half) * (n_seg - 1) + seg) * (DF * D);
+        if (sums_only) S_dst = seg_sums + (((long long)bh * 2 + half) * ((n_seg - 1) * sum_parts) + seg) * (DF * D);
         else if (S_out != nullptr && seg == n_seg - 1) S_dst = S_out + ((long long)bh * NF + half * DF) * D;
         if (S_dst != nullptr) {
             if (n_upd > 0 || has_init) {
@@ -930,20 +947,21 @@ int launch_fused(const still_params_t *p, long long N, const void *Q, const void
     CUtensorMap tq, tw, tk, tv;
     const unsigned long long BH = (unsigned long long)p->B * p->H, BHkv = (unsigned long long)p->B * p->Hkv;
     if (!make_map_2d(&tq, Q, BH * N, D, 128, false) || !make_map_2d(&tw, Wq, (unsigned long long)p->H * D, DF, D, false) ||
-        !make_map_2d(&tk, phiK, BHkv * N, 2 * DF, 64, false) || !make_map_2d(&tv, V, BHkv * N, D, 64, false))
+        !make_map_2d(&tk, phiK, BHkv * N, 2 * DF, FusedPlan<D, DF>::kUTok, false) ||
+        !make_map_2d(&tv, V, BHkv * N, D, FusedPlan<D, DF>::kUTok, false))
         return STILL_ERR_CUDA;
     using Plan = FusedPlan<D, DF>;
     if (ensure_dynamic_smem((const void *)la_fused_kernel<D, DF>, Plan::kTotal) != cudaSuccess) return STILL_ERR_CUDA;
     int seg_chunks = 0;
-    const int n_seg = tc_la_segments(p, N, &seg_chunks);
+    const int n_seg = tc_la_segments(p, N, &seg_chunks), parts = tc_la_sum_parts(seg_chunks);
     for (int pass = n_seg > 1 ? 0 : 1; pass < 2; ++pass) {
         // pass 0 (only with several segments): the sum of every segment's own updates; pass 1: the scan proper
-        dim3 grid((unsigned)BH, 2, (unsigned)(pass == 0 ? n_seg - 1 : n_seg));   // head, feature half, segment
+        dim3 grid((unsigned)BH, 2, (unsigned)(pass == 0 ? (n_seg - 1) * parts : n_seg));   // head, feature half, segment (piece)
         la_fused_kernel<D, DF><<<grid, 384, Plan::kTotal, st>>>(tq, tw, tk, tv, (const bf *)bq, (const bf *)G, sel_idx, zpre,
                                                                (bf *)y_part, d_part, S_out, seg_sums, status, p->H, p->Hkv, (int)N,
                                                                p->chunk, p->topk, p->topk > 0 ? (int)(p->max_salient / p->topk) : 0,
                                                                (long long)BH * N * D, (long long)BH * N,
-                                                               seg_chunks, n_seg, pass == 0 ? 1 : 0);
+                                                               seg_chunks, n_seg, parts, pass == 0 ? 1 : 0);
         ++*launches;
         if (cudaGetLastError() != cudaSuccess) return STILL_ERR_CUDA;
     }
@@ -967,6 +985,11 @@ int tc_la_segments(const still_params_t *p, long long N, int *seg_chunks) {
     sc += sc & 1;
     if (seg_chunks) *seg_chunks = (int)sc;
     return n_seg;
+}
+
+// Pieces per segment in the first pass of the two-level scan (each at least two chunks long).
+int tc_la_sum_parts(int seg_chunks) {
+    return (seg_chunks % 4 == 0 && seg_chunks >= 8) ? 4 : (seg_chunks % 2 == 0 && seg_chunks >= 4) ? 2 : 1;
 }
 
 int tc_la_branch(const still_params_t *p, long long N, const void *Q, const void *K, const void *V, const void *G,

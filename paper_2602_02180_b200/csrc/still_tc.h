@@ -69,6 +69,7 @@ int tc_la_branch(const still_params_t *p, long long N, const void *Q, const void
 // Segments of the two-level state scan for these parameters (1 = plain scan); *seg_chunks = chunks per segment.
 // seg_sums holds (segments - 1) partial states [2 d_f, d] fp32 per (batch, head).
 int tc_la_segments(const still_params_t *p, long long N, int *seg_chunks);
+int tc_la_sum_parts(int seg_chunks);
 
 // ---- decode step ----------------------------------------------------------------------
 size_t step_scratch_bytes(const still_params_t *p, long long capacity);
