@@ -614,18 +614,13 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                            ? sel_idx[((long long)bh * Tn + chunk) * lam + i] - (chunk * C + sub * kUTok) : -1;
             }
         };
-        int cur[4], nxt[4];
-        fetch(warp - 2, cur);
-        for (int nu = warp - 2; nu < n_upd; nu += 2) {
-            fetch(nu + 2, nxt);
+        auto process = [&](int nu, const int (&sel)[4]) {
             const bool leaving = (nu0 + nu) % per_chunk >= su;   // tile of the tokens that leave the salient cache
             // the selected rows of the tile as a 32-bit set
             uint32_t rows = 0u;
 #pragma unroll
             for (int q = 0; q < 4; ++q)
-                if (cur[q] >= 0 && cur[q] < kUTok) rows |= 1u << cur[q];
-#pragma unroll
-            for (int q = 0; q < 4; ++q) cur[q] = nxt[q];
+                if (sel[q] >= 0 && sel[q] < kUTok) rows |= 1u << sel[q];
             rows = __reduce_or_sync(0xffffffffu, rows);
             if (leaving) rows = ~rows;                           // rows to zero: the selected ones, or all the others
             if (ok) ok = mbar_wait(u_full + nu % kUS, (nu / kUS) & 1, abort_flag, status, 67);
@@ -647,6 +642,15 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(u_masked + nu % kUS);
+        };
+        // (two register sets that change roles: a copy from one to the other would wait for the loads)
+        int sel_a[4], sel_b[4];
+        fetch(warp - 2, sel_a);
+        for (int nu = warp - 2; nu < n_upd; nu += 4) {
+            fetch(nu + 2, sel_b);
+            process(nu, sel_a);
+            fetch(nu + 4, sel_a);
+            if (nu + 2 < n_upd) process(nu + 2, sel_b);
         }
     }
     } else if (warp < 8) {
