@@ -352,7 +352,7 @@ struct FusedPlan {
     static constexpr int oZ = oDinv + 8 * 64 * 4;       // [4 map warps][d_f] z half of the chunk two back
     static constexpr int oStage = oZ + 4 * DF * 4;      // [64 tokens][d] bf16: the output of a sub-chunk on its way out
     static constexpr int oBar = oStage + 64 * D * 2;
-    static constexpr int kNumBars = 28;
+    static constexpr int kNumBars = 30;
     static constexpr int oMisc = oBar + kNumBars * 8;
     static constexpr int kTotal = oMisc + 16;
 };
@@ -372,7 +372,8 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     constexpr int NF = 2 * DF;
     extern __shared__ __align__(1024) uint8_t smem[];
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + P::oBar);
-    uint64_t *w_full = bars, *x_full = bars + 1, *x_empty = bars + 2, *f_done = bars + 3, *f_free = bars + 4;
+    uint64_t *w_full = bars, *x_full = bars + 1, *x_empty = bars + 2;
+    uint64_t *f_done = bars + 28, *f_free = bars + 3;   // [2] each: f of even / odd blocks
     uint64_t *pq_full = bars + 5, *pq_empty = bars + 7, *r_done = bars + 9, *out_free = bars + 11, *fin = bars + 13;
     uint64_t *init_done = bars + 14, *u_full = bars + 15, *u_empty = u_full + P::kUStages, *u_masked = u_empty + P::kUStages;
     constexpr int kUS = P::kUStages, kUTok = P::kUTok;
@@ -421,8 +422,10 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         mbar_init(w_full, 1);
         mbar_init(x_full, 1);
         mbar_init(x_empty, 5);      // the f GEMM has read the rows (1) and so have the four map warps (4)
-        mbar_init(f_done, 1);
-        mbar_init(f_free, 4);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(f_done + i, 1);
+            mbar_init(f_free + i, 4);
+        }
         for (int i = 0; i < 2; ++i) {
             mbar_init(pq_full + i, 2);   // the two map warps that own the slot's 64 rows
             mbar_init(pq_empty + i, 1);
@@ -449,7 +452,7 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const uint32_t tmem_base = __shfl_sync(0xffffffffu, *tmem_base_slot, 0);
     // TMEM columns: S^T half [value lanes x d_f features] fp32; f = x W_q of a block [128 rows x d_f]; two read-out
     // results [value lanes x 64 tokens]
-    constexpr uint32_t col_state = 0, col_f = DF, col_out = 2 * DF;
+    constexpr uint32_t col_state = 0, col_f = DF, col_out = 3 * DF;   // f: two buffers of DF columns
 
     // Registers move from the first warpgroup (single-thread roles) to the map warps, whose threads hold a row of f
     // (per scheduler: 72 + 152 + 224 registers for its three warps, of the 3 x 168 the CTA was launched with).
@@ -533,16 +536,16 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             auto issue_f = [&]() {
                 if (nx == 0) wait(w_full, 0, 61);
                 wait(x_full, nx & 1, 62);
-                wait(f_free, (nx & 1) ^ 1, 63);
+                wait(f_free + (nx & 1), ((nx >> 1) & 1) ^ 1, 63);
                 tc_fence_after();
                 if (leader && ok) {
 #pragma unroll
                     for (int k = 0; k < D / 16; ++k) {
                         const uint32_t xo = ((k / 4) * (128 * 128) + (k % 4) * 32) >> 4, wo = (k * (16 * 128)) >> 4;
-                        if (k == 0) mma_ss_lo<idesc_f, 0>(tmem_base + col_f, x_lo + xo, w_lo + wo);
-                        else mma_ss_lo<idesc_f, 1>(tmem_base + col_f, x_lo + xo, w_lo + wo);
+                        if (k == 0) mma_ss_lo<idesc_f, 0>(tmem_base + col_f + (nx & 1) * DF, x_lo + xo, w_lo + wo);
+                        else mma_ss_lo<idesc_f, 1>(tmem_base + col_f + (nx & 1) * DF, x_lo + xo, w_lo + wo);
                     }
-                    tc_commit(f_done);
+                    tc_commit(f_done + (nx & 1));
                     tc_commit(x_empty);
                 }
                 ++nx;
@@ -695,38 +698,41 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             ok = __all_sync(0xffffffffu, ok);
             if (ok) {
                 tc_fence_after();
-                // the result is scaled by 1 / (e . z) of its token here (all loads of the scales come before the first
-                // store below: shared-memory loads are kept behind earlier stores)
+                // y_part[t][e] = N_part / D_part (times the gate): the read-out scaled by 1 / (e . z) of its token.  A thread holds one value column of 64 tokens, but
+                // the rows of y_part are token-major and a store loop over tokens costs about a hundred clocks per
+                // instruction; so the tile is transposed through shared memory and leaves in 16-byte pieces.  Two
+                // rolled rounds of 32 tokens keep the instruction stream short; the scales of a round are loaded
+                // before its first store (shared-memory loads are kept behind earlier stores).
                 const float4 *dinv = reinterpret_cast<const float4 *>(dinv_ring + (u & 7) * 64);
-                uint32_t o[64];
-                tmem_ld32(taddr + col_out + (nq & 1) * 64, o);
-                tmem_ld32(taddr + col_out + (nq & 1) * 64 + 32, o + 32);
-                tmem_wait_ld();
+                __nv_bfloat16 *stg = reinterpret_cast<__nv_bfloat16 *>(smem + P::oStage);
+#pragma unroll 1
+                for (int hf = 0; hf < 2; ++hf) {
+                    uint32_t o[32];
+                    tmem_ld32(taddr + col_out + (nq & 1) * 64 + hf * 32, o);
+                    float4 sc4[8];
 #pragma unroll
-                for (int t4 = 0; t4 < 16; ++t4) {
-                    const float4 sc = dinv[t4];
-                    o[4 * t4] = __float_as_uint(__uint_as_float(o[4 * t4]) * sc.x);
-                    o[4 * t4 + 1] = __float_as_uint(__uint_as_float(o[4 * t4 + 1]) * sc.y);
-                    o[4 * t4 + 2] = __float_as_uint(__uint_as_float(o[4 * t4 + 2]) * sc.z);
-                    o[4 * t4 + 3] = __float_as_uint(__uint_as_float(o[4 * t4 + 3]) * sc.w);
+                    for (int t4 = 0; t4 < 8; ++t4) sc4[t4] = dinv[hf * 8 + t4];
+                    tmem_wait_ld();
+                    if (e < D) {
+#pragma unroll
+                        for (int t4 = 0; t4 < 8; ++t4) {
+                            __nv_bfloat16 *dst = stg + (hf * 32 + 4 * t4) * D + e;
+                            dst[0] = __float2bfloat16_rn(__uint_as_float(o[4 * t4]) * sc4[t4].x);
+                            dst[D] = __float2bfloat16_rn(__uint_as_float(o[4 * t4 + 1]) * sc4[t4].y);
+                            dst[2 * D] = __float2bfloat16_rn(__uint_as_float(o[4 * t4 + 2]) * sc4[t4].z);
+                            dst[3 * D] = __float2bfloat16_rn(__uint_as_float(o[4 * t4 + 3]) * sc4[t4].w);
+                        }
+                    }
                 }
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(out_free + (nq & 1));
-                // y_part[t][e] = N_part / D_part (times the gate).  A thread holds one value column of 64 tokens, but
-                // the rows of y_part are token-major and a store loop over tokens costs about a hundred clocks per
-                // instruction; so the tile is transposed through shared memory and leaves in 16-byte pieces.
-                __nv_bfloat16 *stg = reinterpret_cast<__nv_bfloat16 *>(smem + P::oStage);
-                if (e < D) {
-#pragma unroll
-                    for (int t = 0; t < 64; ++t) stg[t * D + e] = __float2bfloat16_rn(__uint_as_float(o[t]));
-                }
             }
             asm volatile("bar.sync 2, 128;" ::: "memory");   // the four worker warps (always, whatever `ok`)
             if (ok) {
                 const int base = u * 64;
                 constexpr int kPiecesPerRow = D / 8;
-#pragma unroll
+#pragma unroll 2
                 for (int it = 0; it < 64 * kPiecesPerRow / 128; ++it) {
                     const int id = it * 128 + tid, t = id / kPiecesPerRow, c = id % kPiecesPerRow;
                     if (base + t < N) {
@@ -821,26 +827,18 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             __syncwarp();
             if (lane == 0) mbar_arrive(x_empty);
             if (lane < DF / 4) reinterpret_cast<float4 *>(zs)[lane] = zreg;
-            if (ok) ok = mbar_wait(f_done, nx & 1, abort_flag, status, 71);
+            // f of this block is read from tensor memory twice, 32 columns at a time, in loops that stay rolled: the
+            // warp's instruction stream per block is then a few kilobytes.  (With the row held in 128 registers and
+            // everything unrolled, instruction fetch was the first stall reason of the kernel.)  f has a buffer per
+            // block parity, so the next block's GEMM does not wait for this second reading.
+            const uint32_t faddr = taddr + col_f + (nx & 1) * DF;
+            if (ok) ok = mbar_wait(f_done + (nx & 1), (nx >> 1) & 1, abort_flag, status, 71);
             ok = __all_sync(0xffffffffu, ok);
-            float fv[DF];
-            if (ok) {
-                tc_fence_after();
-#pragma unroll
-                for (int q = 0; q < DF / 32; ++q) tmem_ld32(taddr + col_f + q * 32, reinterpret_cast<uint32_t *>(fv) + q * 32);
-                tmem_wait_ld();
-                tc_fence_before();
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(f_free);
             float sgn = 0.f, shift = 0.f;
             if (ok) {
-                // (packed arithmetic and four independent chains each: the row is long and these are latency-bound
-                // reductions; this CTA's half needs only one extremum: max f for softmax(u), min f for softmax(-u))
-                if (bias != nullptr) {
-#pragma unroll
-                    for (int j = 0; j < DF; ++j) fv[j] += __bfloat162float(bias[j]);
-                }
+                tc_fence_after();
+                // (packed arithmetic and four independent chains each; this CTA's half needs only one extremum:
+                // max f for softmax(u), min f for softmax(-u))
                 float2 n2[4];
                 float ex[4];
 #pragma unroll
@@ -848,13 +846,23 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     n2[q] = make_float2(0.f, 0.f);
                     ex[q] = half == 0 ? -INFINITY : INFINITY;
                 }
+#pragma unroll 1
+                for (int q = 0; q < DF / 32; ++q) {
+                    float fv[32];
+                    tmem_ld32(faddr + q * 32, reinterpret_cast<uint32_t *>(fv));
+                    tmem_wait_ld();
+                    if (bias != nullptr) {
 #pragma unroll
-                for (int j = 0; j < DF; j += 8) {
+                        for (int j = 0; j < 32; ++j) fv[j] += __bfloat162float(bias[q * 32 + j]);
+                    }
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const float2 v = make_float2(fv[j + 2 * q], fv[j + 2 * q + 1]);
-                        n2[q] = __ffma2_rn(v, v, n2[q]);
-                        ex[q] = half == 0 ? max3(ex[q], v.x, v.y) : min3(ex[q], v.x, v.y);
+                    for (int j = 0; j < 32; j += 8) {
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            const float2 v = make_float2(fv[j + 2 * c], fv[j + 2 * c + 1]);
+                            n2[c] = __ffma2_rn(v, v, n2[c]);
+                            ex[c] = half == 0 ? max3(ex[c], v.x, v.y) : min3(ex[c], v.x, v.y);
+                        }
                     }
                 }
                 const float nf2 = ((n2[0].x + n2[0].y) + (n2[1].x + n2[1].y)) + ((n2[2].x + n2[2].y) + (n2[3].x + n2[3].y));
@@ -873,23 +881,27 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             if (ok) {
                 // The features go into the tile unnormalised, e_j = 2^(+-u_j - max): with D_part = (e . z) / sum e and
                 // N_part = (e . S) / sum e the output N_part / D_part = (e . S) / (e . z) does not need the sum, so the
-                // row is written as it is computed.  The z values of the next group of 16 features are loaded before
-                // the stores of this group (shared-memory loads are kept behind earlier stores).
+                // row is written as it is computed.  The z values of a block of 32 features are loaded before the
+                // block's stores (shared-memory loads are kept behind earlier stores).
                 uint8_t *tile = smem + P::oQ + slot * P::kPhiQ;
                 float2 zs2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)}, ds2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
                 const float2 sgn2 = make_float2(sgn, sgn), shift2 = make_float2(shift, shift);
-                float4 zc[4];
+#pragma unroll 1
+                for (int q = 0; q < DF / 32; ++q) {          // 32 features: one swizzle atom of the tile
+                    float fv[32];
+                    tmem_ld32(faddr + q * 32, reinterpret_cast<uint32_t *>(fv));
+                    float4 zc[8];
 #pragma unroll
-                for (int i = 0; i < 4; ++i) zc[i] = *reinterpret_cast<const float4 *>(zs + 4 * i);
+                    for (int i = 0; i < 8; ++i) zc[i] = *reinterpret_cast<const float4 *>(zs + 32 * q + 4 * i);
+                    tmem_wait_ld();
+                    if (bias != nullptr) {
 #pragma unroll
-                for (int g = 0; g < DF / 16; ++g) {
-                    float4 zn[4];
+                        for (int j = 0; j < 32; ++j) fv[j] += __bfloat162float(bias[q * 32 + j]);
+                    }
+                    uint8_t *row = tile + q * (64 * 128) + rr * 128;
 #pragma unroll
-                    for (int i = 0; i < 4; ++i)
-                        zn[i] = g + 1 < DF / 16 ? *reinterpret_cast<const float4 *>(zs + 16 * (g + 1) + 4 * i) : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int j = 16 * g + 4 * i;
+                    for (int i = 0; i < 8; ++i) {
+                        const int j = 4 * i;
                         const float2 a0 = __ffma2_rn(make_float2(fv[j], fv[j + 1]), sgn2, shift2);
                         const float2 a1 = __ffma2_rn(make_float2(fv[j + 2], fv[j + 3]), sgn2, shift2);
                         float4 ev;
@@ -901,18 +913,19 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         zs2[1] = __fadd2_rn(zs2[1], make_float2(ev.z, ev.w));
                         ds2[0] = __ffma2_rn(make_float2(ev.x, ev.y), make_float2(zc[i].x, zc[i].y), ds2[0]);
                         ds2[1] = __ffma2_rn(make_float2(ev.z, ev.w), make_float2(zc[i].z, zc[i].w), ds2[1]);
-                        // features j .. j+3: atom j / 32, 16-byte piece (j % 32) / 4, swizzled by the row
-                        *reinterpret_cast<float4 *>(tile + (j >> 5) * (64 * 128) + rr * 128 + ((((j & 31) >> 2) ^ (rr & 7)) << 4)) = ev;
+                        // features 4 i .. 4 i + 3 of the atom: 16-byte piece i, swizzled by the row
+                        *reinterpret_cast<float4 *>(row + ((i ^ (rr & 7)) << 4)) = ev;
                     }
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) zc[i] = zn[i];
                 }
+                tc_fence_before();
                 const float zsum = (zs2[0].x + zs2[0].y) + (zs2[1].x + zs2[1].y), draw = (ds2[0].x + ds2[0].y) + (ds2[1].x + ds2[1].y);
                 const int t = u * 64 + rr;
                 if (t < N) d_out[(long long)bh * N + t] = draw / zsum;     // D_part
                 dinv_ring[(u & 7) * 64 + rr] = draw > 0.f ? 1.f / draw : 0.f;
                 fence_proxy_async();
             }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(f_free + (nx & 1));
             __syncwarp();
             if (lane == 0) mbar_arrive(pq_full + slot);
         }
