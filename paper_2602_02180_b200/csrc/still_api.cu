@@ -58,7 +58,7 @@ static inline bool la_active(const still_params_t *p) { return p->topk < p->chun
 
 // Workspace plan of the prefill.
 struct FwdPlan {
-    size_t status, scores, sel_idx, phiQ, phiK, csum, zpre, segs, nla, dla, ypart, dpart, ksel, vsel, total;
+    size_t status, scores, sel_idx, phiQ, phiK, csum, zpre, segs, nla, dla, ypart, dpart, ksel, vsel, phiKsel, total;
     long long T, sel_rows;  // chunks; rows of the compacted salient K/V per head
     bool la, tc, tc_la;
 };
@@ -106,6 +106,8 @@ static FwdPlan plan_fwd(const still_params_t *p, long long N) {
         if (p->topk < p->chunk) {  // with topk = chunk the salient prefix is K / V itself: no compacted copy
             w.ksel = take(BH * (size_t)w.sel_rows * p->d * es);
             w.vsel = take(BH * (size_t)w.sel_rows * p->d * es);
+            // (with a budget: phi(K) of the selected rows, from which the leaving tokens enter the state)
+            if (w.tc_la && p->max_salient > 0) w.phiKsel = take(BH * (size_t)w.sel_rows * dp * 2);
         }
     }
     w.total = off;
@@ -306,7 +308,7 @@ static int fwd_typed(const still_params_t *p, long long N, const T *Q, const T *
             n_parts = 2;
             rc = tc_la_branch(p, N, Q, K, V, G, Wq, bq, Wk, bk, sel, phiK, reinterpret_cast<float *>(ws + w.csum),
                               reinterpret_cast<float *>(ws + w.zpre), ypart, dpart, reinterpret_cast<float *>(ws + w.segs), S_out,
-                              z_out,
+                              z_out, w.phiKsel ? ws + w.phiKsel : nullptr, w.phiKsel ? ws + w.vsel : nullptr, w.sel_rows,
                               reinterpret_cast<int *>(ws + w.status), st, &g_launches);
             if (rc != STILL_OK) return rc;
         } else {

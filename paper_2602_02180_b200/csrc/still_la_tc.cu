@@ -363,11 +363,12 @@ template <int D, int DF>
 __global__ void __launch_bounds__(384, 1)
 la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_wq,
                 const __grid_constant__ CUtensorMap tm_phik, const __grid_constant__ CUtensorMap tm_v,
+                const __grid_constant__ CUtensorMap tm_phiks, const __grid_constant__ CUtensorMap tm_vs,
                 const __nv_bfloat16 *__restrict__ bq, const __nv_bfloat16 *__restrict__ G,
                 const int32_t *__restrict__ sel_idx, const float *__restrict__ zpre, __nv_bfloat16 *__restrict__ y_part,
                 float *__restrict__ d_part, float *__restrict__ S_out, float *__restrict__ seg_sums, int *status, int H, int Hkv,
                 int N, int C, int lam, int window, long long part_stride_y, long long part_stride_d, int seg_chunks, int n_seg,
-                int sum_parts, int sums_only) {
+                int sum_parts, int sums_only, int sel_rows) {
     using P = FusedPlan<D, DF>;
     constexpr int NF = 2 * DF;
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -402,8 +403,11 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     // Update tiles of kUTok tokens: per routed chunk its su tiles (selected rows zeroed) and, with a salient-cache
     // budget of `window` chunks, the su tiles of the chunk `window` back with everything but its selected rows
     // zeroed: those tokens leave the cache for the state when the chunk is routed.
+    // With sel_rows > 0 the leaving tokens come from the gathered copies of their phi(K) and V rows (sel_rows rows
+    // per head, lam per chunk): nl tiles per chunk instead of su, and only a last partial tile has rows to clear.
     const int su = C / kUTok;
-    const int per_chunk = window > 0 ? 2 * su : su;
+    const int nl = sel_rows > 0 ? (lam + kUTok - 1) / kUTok : su;
+    const int per_chunk = window > 0 ? su + nl : su;
     const int nu0 = (u_first / sc - 2) * per_chunk;    // first update tile of the segment
     const int n_upd = NU > u_first ? ((NU - 1) / sc - 1) * per_chunk - nu0 : 0;
     const bool has_init = !sums_only && seg > 0;
@@ -484,12 +488,15 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     // `window` back (before there is one, any valid tile: all its rows are zeroed)
                     const int a_t = nu0 + nu, cc = a_t / per_chunk, rt = a_t % per_chunk;
                     const int src = (rt >= su && cc >= window) ? cc - window : cc;
-                    const int tile_sub = src * su + rt % su;
+                    const bool gathered = rt >= su && sel_rows > 0;
+                    // first row of the tile: in phi(K) / V of the KV head, or in the head's gathered rows
+                    const int row = gathered ? bh * sel_rows + src * lam + (rt - su) * kUTok : kv_row0 + (src * su + rt % su) * kUTok;
+                    const CUtensorMap *mp = gathered ? &tm_phiks : &tm_phik, *mv = gathered ? &tm_vs : &tm_v;
                     mbar_expect_tx(u_full + nu % kUS, P::kUStage);
                     for (int a = 0; a < DF / 64; ++a)  // phi(K) half: MN-major, 64-feature atoms kUTok rows apart
-                        tma_load_2d(stg + a * (kUTok * 128), &tm_phik, u_full + nu % kUS, half * DF + a * 64, kv_row0 + tile_sub * kUTok);
+                        tma_load_2d(stg + a * (kUTok * 128), mp, u_full + nu % kUS, half * DF + a * 64, row);
                     for (int a = 0; a < D / 64; ++a)   // V: M-major A operand, 64-column atoms kUTok rows apart
-                        tma_load_2d(stg + P::kPhiK + a * (kUTok * 128), &tm_v, u_full + nu % kUS, a * 64, kv_row0 + tile_sub * kUTok);
+                        tma_load_2d(stg + P::kPhiK + a * (kUTok * 128), mv, u_full + nu % kUS, a * 64, row);
                     ++nu;
                     progressed = true;
                 }
@@ -610,15 +617,17 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         auto fetch = [&](int nu, int (&r)[4]) {
             const int a_t = nu0 + nu, cc = a_t / per_chunk, rt = a_t % per_chunk, sub = rt % su;
             const int chunk = rt >= su ? cc - window : cc;       // (chunk < 0: nothing leaves yet, every row is zeroed)
+            const bool need = !(rt >= su && sel_rows > 0);       // (a gathered tile needs no indices)
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
                 const int i = lane + 32 * q;
-                r[q] = (nu < n_upd && i < lam && chunk >= 0)
+                r[q] = (need && nu < n_upd && i < lam && chunk >= 0)
                            ? sel_idx[((long long)bh * Tn + chunk) * lam + i] - (chunk * C + sub * kUTok) : -1;
             }
         };
         auto process = [&](int nu, const int (&sel)[4]) {
-            const bool leaving = (nu0 + nu) % per_chunk >= su;   // tile of the tokens that leave the salient cache
+            const int rt = (nu0 + nu) % per_chunk;
+            const bool leaving = rt >= su;                       // tile of the tokens that leave the salient cache
             // the selected rows of the tile as a 32-bit set
             uint32_t rows = 0u;
 #pragma unroll
@@ -626,6 +635,12 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 if (sel[q] >= 0 && sel[q] < kUTok) rows |= 1u << sel[q];
             rows = __reduce_or_sync(0xffffffffu, rows);
             if (leaving) rows = ~rows;                           // rows to zero: the selected ones, or all the others
+            if (leaving && sel_rows > 0) {
+                // gathered tile: its first `valid` rows are the chunk's leaving tokens, the rest belong to the next chunk
+                const int cw = (nu0 + nu) / per_chunk - window;
+                const int valid = cw < 0 ? 0 : min(kUTok, lam - (rt - su) * kUTok);
+                rows = valid >= 32 ? 0u : ~((1u << valid) - 1u);
+            }
             if (ok) ok = mbar_wait(u_full + nu % kUS, (nu / kUS) & 1, abort_flag, status, 67);
             ok = __all_sync(0xffffffffu, ok);
             if (ok) {
@@ -938,6 +953,32 @@ la_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     }
 }
 
+// Rows of phi(K) [2 d_f] and V [d] of the selected tokens, per query head, in selection order (row j of a head is
+// token sel_idx[j]; -1 entries and the padding up to sel_rows are zero): with a salient-cache budget the tokens
+// that leave the cache enter the state from these copies, lam rows per chunk.  One warp per row.
+template <int D, int DF>
+__global__ void __launch_bounds__(256)
+gather_selected_kernel(const __nv_bfloat16 *__restrict__ phiK, const __nv_bfloat16 *__restrict__ V,
+                       const int32_t *__restrict__ sel_idx, __nv_bfloat16 *__restrict__ phiKsel,
+                       __nv_bfloat16 *__restrict__ Vsel, int H, int Hkv, long long N, long long n_idx, long long sel_rows) {
+    const int bh = blockIdx.y, b = bh / H, h = bh % H, kvh = h / (H / Hkv);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long j = (long long)blockIdx.x * 8 + warp;
+    if (j >= sel_rows) return;
+    long long pos = -1;
+    if (j < n_idx) pos = sel_idx[(long long)bh * n_idx + j];
+    constexpr int kPhiVec = 2 * DF / 8, kVVec = D / 8;   // uint4 per row
+    uint4 pp = make_uint4(0, 0, 0, 0), vv = pp;
+    const long long src = ((long long)b * Hkv + kvh) * N + pos;
+    if (pos >= 0) {
+        if (lane < kPhiVec) pp = reinterpret_cast<const uint4 *>(phiK + src * (2 * DF))[lane];
+        if (lane < kVVec) vv = reinterpret_cast<const uint4 *>(V + src * D)[lane];
+    }
+    const long long dst = (long long)bh * sel_rows + j;
+    if (lane < kPhiVec) reinterpret_cast<uint4 *>(phiKsel + dst * (2 * DF))[lane] = pp;
+    if (lane < kVVec) reinterpret_cast<uint4 *>(Vsel + dst * D)[lane] = vv;
+}
+
 // ------------------------------------------------------------------------------------------ host side
 
 template <int D, int DF, typename TOut>
@@ -959,14 +1000,32 @@ int launch_npmap(const void *X, const void *W, const void *bias, void *phi, floa
 template <int D, int DF>
 int launch_fused(const still_params_t *p, long long N, const void *Q, const void *V, const void *G, const void *Wq,
                  const void *bq, const int32_t *sel_idx, const void *phiK, const float *zpre, void *y_part, float *d_part,
-                 float *S_out, float *seg_sums, int *status, cudaStream_t st, int *launches) {
+                 float *S_out, float *seg_sums, void *phiK_sel, void *v_sel, long long sel_rows, int *status, cudaStream_t st,
+                 int *launches) {
     using bf = __nv_bfloat16;
-    CUtensorMap tq, tw, tk, tv;
+    CUtensorMap tq, tw, tk, tv, tks, tvs;
     const unsigned long long BH = (unsigned long long)p->B * p->H, BHkv = (unsigned long long)p->B * p->Hkv;
     if (!make_map_2d(&tq, Q, BH * N, D, 128, false) || !make_map_2d(&tw, Wq, (unsigned long long)p->H * D, DF, D, false) ||
         !make_map_2d(&tk, phiK, BHkv * N, 2 * DF, FusedPlan<D, DF>::kUTok, false) ||
         !make_map_2d(&tv, V, BHkv * N, D, FusedPlan<D, DF>::kUTok, false))
         return STILL_ERR_CUDA;
+    // With a salient-cache budget and topk < chunk the leaving tokens are read from gathered copies of their rows
+    // (otherwise every token of a chunk is selected and the chunk's own tiles are the leaving tiles).
+    const bool gathered = p->max_salient > 0 && p->topk < p->chunk && phiK_sel != nullptr && v_sel != nullptr;
+    tks = tk;
+    tvs = tv;
+    if (gathered) {
+        if (BH * (unsigned long long)sel_rows >= (1ull << 31)) return STILL_ERR_UNSUPPORTED;   // TMA row coordinate
+        const long long Tn = (N + p->chunk - 1) / p->chunk;
+        dim3 ggrid((unsigned)((sel_rows + 7) / 8), (unsigned)BH);
+        gather_selected_kernel<D, DF><<<ggrid, 256, 0, st>>>((const bf *)phiK, (const bf *)V, sel_idx, (bf *)phiK_sel, (bf *)v_sel,
+                                                           p->H, p->Hkv, N, Tn * p->topk, sel_rows);
+        ++*launches;
+        if (cudaGetLastError() != cudaSuccess) return STILL_ERR_CUDA;
+        if (!make_map_2d(&tks, phiK_sel, BH * (unsigned long long)sel_rows, 2 * DF, FusedPlan<D, DF>::kUTok, false) ||
+            !make_map_2d(&tvs, v_sel, BH * (unsigned long long)sel_rows, D, FusedPlan<D, DF>::kUTok, false))
+            return STILL_ERR_CUDA;
+    }
     using Plan = FusedPlan<D, DF>;
     if (ensure_dynamic_smem((const void *)la_fused_kernel<D, DF>, Plan::kTotal) != cudaSuccess) return STILL_ERR_CUDA;
     int seg_chunks = 0;
@@ -974,11 +1033,11 @@ int launch_fused(const still_params_t *p, long long N, const void *Q, const void
     for (int pass = n_seg > 1 ? 0 : 1; pass < 2; ++pass) {
         // pass 0 (only with several segments): the sum of every segment's own updates; pass 1: the scan proper
         dim3 grid((unsigned)BH, 2, (unsigned)(pass == 0 ? (n_seg - 1) * parts : n_seg));   // head, feature half, segment (piece)
-        la_fused_kernel<D, DF><<<grid, 384, Plan::kTotal, st>>>(tq, tw, tk, tv, (const bf *)bq, (const bf *)G, sel_idx, zpre,
+        la_fused_kernel<D, DF><<<grid, 384, Plan::kTotal, st>>>(tq, tw, tk, tv, tks, tvs, (const bf *)bq, (const bf *)G, sel_idx, zpre,
                                                                (bf *)y_part, d_part, S_out, seg_sums, status, p->H, p->Hkv, (int)N,
                                                                p->chunk, p->topk, p->topk > 0 ? (int)(p->max_salient / p->topk) : 0,
                                                                (long long)BH * N * D, (long long)BH * N,
-                                                               seg_chunks, n_seg, parts, pass == 0 ? 1 : 0);
+                                                               seg_chunks, n_seg, parts, pass == 0 ? 1 : 0, gathered ? (int)sel_rows : 0);
         ++*launches;
         if (cudaGetLastError() != cudaSuccess) return STILL_ERR_CUDA;
     }
@@ -1012,7 +1071,7 @@ int tc_la_sum_parts(int seg_chunks) {
 int tc_la_branch(const still_params_t *p, long long N, const void *Q, const void *K, const void *V, const void *G,
                  const void *Wq, const void *bq, const void *Wk, const void *bk, const int32_t *sel_idx, void *phiK,
                  float *csum, float *zpre, void *y_part, float *d_part, float *seg_sums, float *S_out, float *z_out,
-                 int *status_words, cudaStream_t st, int *launches) {
+                 void *phiK_sel, void *v_sel, long long sel_rows, int *status_words, cudaStream_t st, int *launches) {
     using bf = __nv_bfloat16;
     if ((long long)p->B * p->H * N >= (1ll << 31)) return STILL_ERR_UNSUPPORTED;  // TMA row coordinate
     const int NF = 2 * p->d_f, C = p->chunk;
@@ -1041,10 +1100,13 @@ int tc_la_branch(const still_params_t *p, long long N, const void *Q, const void
         if (cudaGetLastError() != cudaSuccess) return STILL_ERR_CUDA;
     }
     if (p->d == 64 && p->d_f == 64)
-        return launch_fused<64, 64>(p, N, Q, V, G, Wq, bq, sel_idx, phiK, zpre, y_part, d_part, S_out, seg_sums, status_words, st, launches);
+        return launch_fused<64, 64>(p, N, Q, V, G, Wq, bq, sel_idx, phiK, zpre, y_part, d_part, S_out, seg_sums, phiK_sel, v_sel, sel_rows,
+                                   status_words, st, launches);
     if (p->d == 128 && p->d_f == 64)
-        return launch_fused<128, 64>(p, N, Q, V, G, Wq, bq, sel_idx, phiK, zpre, y_part, d_part, S_out, seg_sums, status_words, st, launches);
-    return launch_fused<128, 128>(p, N, Q, V, G, Wq, bq, sel_idx, phiK, zpre, y_part, d_part, S_out, seg_sums, status_words, st, launches);
+        return launch_fused<128, 64>(p, N, Q, V, G, Wq, bq, sel_idx, phiK, zpre, y_part, d_part, S_out, seg_sums, phiK_sel, v_sel, sel_rows,
+                                   status_words, st, launches);
+    return launch_fused<128, 128>(p, N, Q, V, G, Wq, bq, sel_idx, phiK, zpre, y_part, d_part, S_out, seg_sums, phiK_sel, v_sel, sel_rows,
+                                   status_words, st, launches);
 }
 
 }  // namespace still

@@ -65,7 +65,7 @@ bool tc_la_supported(const still_params_t *p);
 int tc_la_branch(const still_params_t *p, long long N, const void *Q, const void *K, const void *V, const void *G,
                  const void *Wq, const void *bq, const void *Wk, const void *bk, const int32_t *sel_idx, void *phiK,
                  float *csum, float *zpre, void *y_part, float *d_part, float *seg_sums, float *S_out, float *z_out,
-                 int *status_words, cudaStream_t st, int *launches);
+                 void *phiK_sel, void *v_sel, long long sel_rows, int *status_words, cudaStream_t st, int *launches);
 // Segments of the two-level state scan for these parameters (1 = plain scan); *seg_chunks = chunks per segment.
 // seg_sums holds (segments - 1) partial states [2 d_f, d] fp32 per (batch, head).
 int tc_la_segments(const still_params_t *p, long long N, int *seg_chunks);
