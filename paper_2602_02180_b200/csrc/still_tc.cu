@@ -177,15 +177,9 @@ __device__ __forceinline__ void softmax_role(const StreamT &st, const int x, con
             tmem_wait_ld();
             float *s = reinterpret_cast<float *>(sr);
             if (need_mask) {
-                // per block of 32 columns: nothing to do where every row of the warp sees the whole block
 #pragma unroll
-                for (int ch = 0; ch < 4; ++ch) {
-                    if (!__all_sync(0xffffffffu, lo <= 32 * ch && hi >= 32 * ch + 31)) {
-#pragma unroll
-                        for (int j = 32 * ch; j < 32 * ch + 32; ++j)
-                            if (j < lo || j > hi) s[j] = -INFINITY;
-                    }
-                }
+                for (int j = 0; j < 128; ++j)
+                    if (j < lo || j > hi) s[j] = -INFINITY;
             }
             float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
@@ -259,38 +253,18 @@ __device__ __forceinline__ void softmax_role(const StreamT &st, const int x, con
         // warp's 32 rows of the tile's Q region (one row = D bf16 = 2 D bytes: D / 2 columns of both parts), free
         // once the tile's last Q K^T has completed; 16-byte pieces are swizzled by the row so that row-wise and
         // piece-wise accesses avoid bank conflicts.
-        // The partial results are requested before the wait for the tile's last P V product (first half) and while
-        // the first half is being merged (second half), so that their way from memory lies under other work.
-        constexpr int kRowBytes = D * 2, kPieces = kRowBytes / 16;   // pieces of 16 bytes per staged row
-        constexpr int kPartPieces = kPieces / 2;                     // pieces of one part (D / 2 columns)
-        const int t0 = tile_row0 + (warp & 3) * 32;                    // first row of this warp
-        auto load_parts = [&](int hh, uint4 (&v)[kPieces]) {
-#pragma unroll
-            for (int it = 0; it < kPieces; ++it) {
-                const int id = it * 32 + lane, row = id / kPieces, c = id % kPieces;
-                const int part = c / kPartPieces, cc = c % kPartPieces;
-                v[it] = make_uint4(0, 0, 0, 0);
-                if (t0 + row < N && part < n_parts)
-                    v[it] = *reinterpret_cast<const uint4 *>(y_part + part * part_stride_y + ((long long)bh * N + t0 + row) * D +
-                                                             hh * (D / 2) + cc * 8);
-            }
-        };
-        uint4 pre[kPieces];
-        float da = 0.f, db = 0.f;
-        if (n_parts > 0) {
-            if (t < N) {
-                da = d_part[(long long)bh * N + t];
-                db = n_parts > 1 ? d_part[part_stride_d + (long long)bh * N + t] : 0.f;
-            }
-            load_parts(0, pre);
-        }
         if (ok) ok = mbar_wait(o_final + x, 0, abort_flag, status, 9);
         ok = __all_sync(0xffffffffu, ok);
         if (ok) {
             tc_fence_after();
+            constexpr int kRowBytes = D * 2, kPieces = kRowBytes / 16;   // pieces of 16 bytes per staged row
+            constexpr int kPartPieces = kPieces / 2;                     // pieces of one part (D / 2 columns)
             uint8_t *stg = stage_tile + (warp & 3) * 32 * kRowBytes;
+            const int t0 = tile_row0 + (warp & 3) * 32;                    // first row of this warp
             float fs = 1.f, fa = 0.f, fb = 0.f, dla = 0.f;
             if (n_parts > 0 && t < N) {
+                const float da = d_part[(long long)bh * N + t];
+                const float db = n_parts > 1 ? d_part[part_stride_d + (long long)bh * N + t] : 0.f;
                 dla = da + db;
                 if (dla > 0.f) {
                     const float m_nat = m_used * 0.6931471805599453f;
@@ -311,9 +285,13 @@ __device__ __forceinline__ void softmax_role(const StreamT &st, const int x, con
 #pragma unroll
                     for (int it = 0; it < kPieces; ++it) {
                         const int id = it * 32 + lane, row = id / kPieces, c = id % kPieces;
-                        *reinterpret_cast<uint4 *>(stg + row * kRowBytes + ((c ^ (row & (kPieces - 1))) << 4)) = pre[it];
+                        const int part = c / kPartPieces, cc = c % kPartPieces;
+                        uint4 v = make_uint4(0, 0, 0, 0);
+                        if (t0 + row < N && part < n_parts)
+                            v = *reinterpret_cast<const uint4 *>(y_part + part * part_stride_y + ((long long)bh * N + t0 + row) * D +
+                                                                 hh * (D / 2) + cc * 8);
+                        *reinterpret_cast<uint4 *>(stg + row * kRowBytes + ((c ^ (row & (kPieces - 1))) << 4)) = v;
                     }
-                    if (hh == 0) load_parts(1, pre);
                     __syncwarp();
                 }
 #pragma unroll
